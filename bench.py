@@ -31,14 +31,17 @@ L2_FLUSH_BYTES = 256 << 20
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, help="workload index (2 = QuartzNet-15x5 shape, B=32, T=1600)")
     ap.add_argument("--variant", default="live", choices=["live", "literal"])
     ap.add_argument("--profile-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sustained-seconds", type=float, default=2.0,
+                    help="length of the back-to-back replay run reported as `sustained` (0 = skip)")
+    ap.add_argument("--no-int8-peak", action="store_true", help="skip the tcgen05 int8 saturation loop")
     ap.add_argument("--static-weights", action="store_true",
                     help="promise the library that weights do not change between steps (K-tap layers then keep their regrouped weights)")
     return ap.parse_args()
@@ -52,6 +55,10 @@ def measured_peaks():
         return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
                 "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+NOMINAL_INT8_TOPS = 4500.0      # dense int8, datasheet figure without sparsity
+NOMINAL_HBM_GBS = 7700.0        # HGX B200 datasheet figure
 
 
 class ClockSampler:
@@ -100,7 +107,7 @@ class ClockSampler:
             self.proc.kill()
             out, _ = self.proc.communicate()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        rows = []
+        rows = self.rows = []
         for line in out.splitlines():
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 7:
@@ -111,8 +118,13 @@ class ClockSampler:
                 continue
             active = [nm for nm, v in zip(names, parts[3:7]) if v.lower().startswith("active")]
             rows.append((self._stamp(parts[7]) if len(parts) > 7 else None, row, active))
-        inside = [r for r in rows if r[0] is not None and self.t_begin is not None and self.t_end is not None
-                  and self.t_begin - 0.02 <= r[0] <= self.t_end + 0.02]
+        return self.window(self.t_begin, self.t_end)
+
+    def window(self, t_begin, t_end):
+        """Statistics of the samples stamped inside [t_begin, t_end] (after stop())."""
+        rows = getattr(self, "rows", [])
+        inside = [r for r in rows if r[0] is not None and t_begin is not None and t_end is not None
+                  and t_begin - 0.02 <= r[0] <= t_end + 0.02]
         use = inside if inside else rows          # no stamp inside the window: everything seen while the job ran
         sm = [r[1][0] for r in use]
         mx = [r[1][1] for r in use]
@@ -171,7 +183,9 @@ def run_reference(args):
 # --------------------------------------------------------------------------------------------
 # our arm
 # --------------------------------------------------------------------------------------------
-TENSOR_KERNELS = ("conv_generic", "gemm_i8_tc", "conv_i8_tc", "tcs_fused")
+TENSOR_KERNELS = ("conv_generic", "gemm_i8_tc", "conv_i8_tc")
+DEPTHWISE_KERNELS = ("dw_conv_tc", "dw_conv_dp4a", "dw_conv_generic")
+ELEMENTWISE_KERNELS = ("residual_add", "glu", "dequant", "conv_tc_prepare")
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, averaged over the launches of one step of
 # this workload, caches left as the step leaves them) from the ncu capture summarised in
@@ -253,7 +267,8 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     def timed(fn, steps):
-        """K steps, each between its own pair of events; the L2 flush between steps is outside them."""
+        """K steps, each between its own pair of events; the L2 flush between steps is outside them.
+        Returns (sum of the step times, list of step times), both as the slowest rank's."""
         e0 = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
         e1 = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
         barrier()
@@ -263,26 +278,64 @@ def run_ours(args):
             fn()
             e1[i].record()
         barrier()
-        ms = sum(a.elapsed_time(b) for a, b in zip(e0, e1))
-        return max_over_ranks(ms, world, dev)
+        per = [a.elapsed_time(b) for a, b in zip(e0, e1)]
+        return max_over_ranks(sum(per), world, dev), per
 
     step = lambda: ctx.encoder_forward(dm, xd, ws, lq, lf)
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+
+    # the int8 tensor-core peak of this GPU, from the library's own saturation loop (before the timed region)
+    int8_peak = None
+    if not args.no_int8_peak:
+        burst = max(ctx.measure_int8_tensor_peak(2000)[0] for _ in range(3))       # ~0.5 ms each
+        long_run = ctx.measure_int8_tensor_peak(400000)[0]                         # ~0.1 s: clocks settle under power
+        int8_peak = {"burst_tops": burst, "long_run_tops": long_run,
+                     "how": "tcgen05.mma kind::i8 M=128 N=256 K=32 back to back on every SM, operands fixed in shared "
+                            "memory; burst = best of three 0.5 ms runs, long_run = one run of 400 000 K blocks"}
+
     for _ in range(args.warmup):
         step()
     ctx.poll_status()
 
     n0 = ctx.launch_count()
     sampler.mark_begin()
-    total_ms = timed(step, args.steps)
+    total_ms, per_step = timed(step, args.steps)
     sampler.mark_end()
     launches = ctx.launch_count() - n0
-    clocks = sampler.stop() if rank == 0 else None
     ctx.poll_status()
     frames = world * B * T * args.steps
     value = job_throughput(world, B * T, args.steps, total_ms)
+
+    # sustained: back-to-back replays for a few seconds inside ONE pair of events (no flush: the working set
+    # of a step, ~70 MB of activations + 19 MB of weights, is L2-resident either way; what changes is power)
+    sustained = None
+    sus_window = None
+    if args.sustained_seconds > 0:
+        n_rep = max(10, int(args.sustained_seconds * 1e3 / (total_ms / args.steps)))
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        barrier()
+        t_b = time.time()
+        e0.record()
+        for _ in range(n_rep):
+            step()
+        e1.record()
+        barrier()
+        t_e = time.time()
+        sus_ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
+        sus_window = (t_b, t_e)
+        sustained = {"value": job_throughput(world, B * T, n_rep, sus_ms), "unit": UNIT, "steps": n_rep,
+                     "seconds": sus_ms / 1e3, "ms_per_step": sus_ms / n_rep,
+                     "note": "graph replays back to back inside one event pair, no L2 flush between them"}
+        ctx.poll_status()
+    clocks = sampler.stop() if rank == 0 else None
+    if rank == 0 and sustained is not None:
+        w = sampler.window(*sus_window)
+        sustained["clocks"] = w
+        if w["sm_mhz"] and w["sm_max_mhz"]:
+            sustained["value_scaled_to_max_clock"] = sustained["value"] * w["sm_max_mhz"] / w["sm_mhz"]
 
     # end to end through the host-buffer entry point: pinned host input -> device, forward, logits -> host
     e2e = None
@@ -291,11 +344,13 @@ def run_ours(args):
         lqh = torch.zeros(lq.shape, dtype=torch.int32).pin_memory()
         lfh = torch.zeros(lf.shape, dtype=torch.float32).pin_memory()
         hstep = lambda: ctx.encoder_forward_host(dm, xh, ws, lqh, lfh)
-        for _ in range(max(3, args.warmup)):
+        for _ in range(max(3, min(args.warmup, 5))):
             hstep()
-        e2e_ms = timed(hstep, args.steps)
-        e2e = {"value": frames / (e2e_ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": int(xh.numel()),
-               "d2h_bytes_per_step": int(lqh.numel() * 4 + lfh.numel() * 4), "ms_per_step": e2e_ms / args.steps}
+        e2e_steps = min(args.steps, 30)
+        e2e_ms, _ = timed(hstep, e2e_steps)
+        e2e = {"value": world * B * T * e2e_steps / (e2e_ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": int(xh.numel()),
+               "d2h_bytes_per_step": int(lqh.numel() * 4 + lfh.numel() * 4), "ms_per_step": e2e_ms / e2e_steps,
+               "steps": e2e_steps}
 
     # per-kernel durations: the same step launched kernel by kernel between CUDA events
     kernels = {}
@@ -324,47 +379,71 @@ def run_ours(args):
         return
 
     peaks = measured_peaks()
+    step_ms = total_ms / args.steps
+    tot_kernel_ms = sum(k["ms"] for k in kernels.values()) if kernels else 0.0
+
+    def tensor_roofline(names, label):
+        """Tensor-core roofline of the launches of the given kernels taken together."""
+        ks = [kernels[n] for n in names if n in kernels]
+        if not ks:
+            return None
+        ms = sum(k["ms"] for k in ks)
+        ops = 2 * sum(k["macs"] for k in ks)
+        n_l = sum(k["launches"] for k in ks)
+        ach = ops / (ms * 1e-3) / 1e12
+        two_bf16 = 2.0 * peaks["bf16_tflops"]
+        peak = int8_peak["burst_tops"] if int8_peak else two_bf16
+        share = ms / tot_kernel_ms
+        in_step = ops / args.profile_steps / 1e12 / (share * step_ms * 1e-3)
+        return {"bound": "tensor", "kernel": label, "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
+                "traffic": recorded_traffic(label, args.config),
+                "algorithmic_bytes_per_launch": sum(k["bytes"] for k in ks) / n_l,
+                "launches_per_step": n_l // args.profile_steps,
+                "peak_source": ("measured: the library's tcgen05 kind::i8 saturation loop on this GPU, burst"
+                                if int8_peak else "2 x %s bf16 burst (no int8 loop was run)" % peaks["source"]),
+                "frac_of_2x_%s_bf16_burst" % peaks["source"]: ach / two_bf16,
+                "frac_of_nominal_dense_int8_4500": ach / NOMINAL_INT8_TOPS,
+                "achieved_in_timed_step": in_step, "frac_in_timed_step": in_step / peak,
+                "frac_in_timed_step_of_nominal_dense_int8_4500": in_step / NOMINAL_INT8_TOPS,
+                "note": "int8 multiply-accumulate counted as 2 ops (unit reads TOP/s); achieved = ops of these launches / "
+                        "their CUDA-event time in a kernel-by-kernel pass of the same step; *_in_timed_step: the same "
+                        "work over these kernels' share of the graph-replayed, timed step"}
+
+    def hbm_roofline(names, label):
+        ks = [kernels[n] for n in names if n in kernels]
+        if not ks:
+            return None
+        ms = sum(k["ms"] for k in ks)
+        nbytes = sum(k["bytes"] for k in ks)
+        n_l = sum(k["launches"] for k in ks)
+        ach = nbytes / (ms * 1e-3) / 1e9
+        share = ms / tot_kernel_ms
+        in_step = nbytes / args.profile_steps / 1e9 / (share * step_ms * 1e-3)
+        return {"bound": "hbm", "kernel": label, "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": ach / peaks["hbm_gbs"], "traffic": recorded_traffic(label, args.config),
+                "algorithmic_bytes_per_launch": nbytes / n_l, "launches_per_step": n_l // args.profile_steps,
+                "peak_source": peaks["source"] + " copy bandwidth",
+                "frac_of_nominal_hbm_7700": ach / NOMINAL_HBM_GBS,
+                "achieved_in_timed_step": in_step, "frac_in_timed_step": in_step / peaks["hbm_gbs"],
+                "note": "algorithmic bytes (tensors read + written once) / CUDA-event time in a kernel-by-kernel pass of "
+                        "the same step; the tensors are L2-resident between layers, so this is not DRAM traffic"}
+
     roofline = None
+    roofline_by_kind = {}
     ksum = {}
     if kernels:
-        tot = sum(k["ms"] for k in kernels.values())
         for name, k in kernels.items():
             ksum[name] = {"launches_per_step": k["launches"] // args.profile_steps,
-                          "ms_per_step": k["ms"] / args.profile_steps, "share": k["ms"] / tot,
+                          "ms_per_step": k["ms"] / args.profile_steps, "share": k["ms"] / tot_kernel_ms,
                           "tops": 2 * k["macs"] / (k["ms"] * 1e-3) / 1e12 if k["macs"] else None,
                           "gbs": k["bytes"] / (k["ms"] * 1e-3) / 1e9}
         top = max(kernels, key=lambda n: kernels[n]["ms"])
-        k = kernels[top]
-        if top in TENSOR_KERNELS:
-            peak = 2.0 * peaks["bf16_tflops"]   # dense int8 is nominally 2x the bf16 rate
-            ach = 2 * k["macs"] / (k["ms"] * 1e-3) / 1e12
-            roofline = {"bound": "tensor", "kernel": top, "achieved": ach, "peak": peak, "unit": "TFLOP/s",
-                        "frac": ach / peak, "traffic": recorded_traffic(top, args.config),
-                        "algorithmic_bytes_per_launch": k["bytes"] / k["launches"],
-                        "peak_source": "2 x %s bf16 burst (int8 dense is nominally twice bf16)" % peaks["source"],
-                        "note": "int8 multiply-accumulate counted as 2 ops; per-launch average over %d launches per step, "
-                                "timed kernel by kernel with CUDA events in a separate pass of the same step" % (k["launches"] // args.profile_steps)}
-        else:
-            ach = k["bytes"] / (k["ms"] * 1e-3) / 1e9
-            roofline = {"bound": "hbm", "kernel": top, "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                        "frac": ach / peaks["hbm_gbs"], "traffic": recorded_traffic(top, args.config),
-                        "algorithmic_bytes_per_launch": k["bytes"] / k["launches"],
-                        "peak_source": peaks["source"] + " copy bandwidth",
-                        "note": "algorithmic bytes (tensors read + written once); timed kernel by kernel with CUDA events "
-                                "in a separate pass of the same step"}
-
-    if roofline:
-        # The kernel-by-kernel pass brackets every launch with two events, which keeps a kernel's prologue from
-        # overlapping its predecessor's tail and adds the events' own time. The same kernel's share of the
-        # graph-replayed, timed step is reported beside it: its share of the kernel-by-kernel pass (the ncu
-        # launch list gives the same shares) times the timed step.
-        k = kernels[roofline["kernel"]]
-        share = k["ms"] / sum(v["ms"] for v in kernels.values())
-        in_step_ms = share * (total_ms / args.steps)
-        work = (2 * k["macs"] / args.profile_steps / 1e12) if roofline["bound"] == "tensor" else (k["bytes"] / args.profile_steps / 1e9)
-        roofline["achieved_in_timed_step"] = work / (in_step_ms * 1e-3)
-        roofline["frac_in_timed_step"] = roofline["achieved_in_timed_step"] / roofline["peak"]
-        roofline["note"] += "; *_in_timed_step: the same work over this kernel's share of the graph-replayed step"
+        roofline = tensor_roofline([top], top) if top in TENSOR_KERNELS else hbm_roofline([top], top)
+        roofline_by_kind["pointwise_and_dense_gemm"] = tensor_roofline(
+            [n for n in kernels if n in TENSOR_KERNELS], "all convolution kernels")
+        roofline_by_kind["depthwise"] = hbm_roofline([n for n in kernels if n in DEPTHWISE_KERNELS], "all depthwise kernels")
+        roofline_by_kind["elementwise"] = hbm_roofline([n for n in kernels if n in ELEMENTWISE_KERNELS], "residual add, GLU, dequant, layout kernels")
+    roofline_depthwise = roofline_by_kind.get("depthwise")
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
@@ -381,7 +460,8 @@ def run_ours(args):
                "sample": "%d of %d utterances, full length T=%d, one pass (%.1f s)" % (Bs, B, T, dt)}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": step_ms, "ms_per_step_median": statistics.median(per_step),
+            "ms_per_step_min": min(per_step), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int8", "data": "synthetic",
             "config": {"workload": "config %d: %s B=%d T=%d mel=%d (%s scales)" % (args.config, model["name"], B, T, C_in, args.variant),
                        "per_gpu_batch": B, "layers": len(model["layers"]),
@@ -389,6 +469,10 @@ def run_ours(args):
                        "static_weights": bool(args.static_weights),
                        "parallelism": "replicas x%d, no collective" % world},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+            "roofline_depthwise": roofline_depthwise, "roofline_by_kind": roofline_by_kind,
+            "int8_peak": int8_peak, "sustained": sustained,
+            "peaks": {"hbm_gbs": peaks["hbm_gbs"], "bf16_tflops": peaks["bf16_tflops"], "source": peaks["source"],
+                      "nominal_dense_int8_tops": NOMINAL_INT8_TOPS, "nominal_hbm_gbs": NOMINAL_HBM_GBS},
             "cpu_baseline": cpu, "kernels": ksum}
     print(json.dumps(line))
     if world > 1:

@@ -123,6 +123,23 @@ const char* qasr_kernel_name(int kernel);
 /* Number of kernels this context has launched (graph replays count their kernel nodes). */
 int64_t qasr_launch_count(const qasr_ctx* ctx);
 
+/* Diagnostic: checks the library's own failure detection.  Every wait inside the tensor-core kernels
+ * (on a TMA copy, on the tensor pipe, on a free buffer) is bounded; when one expires the kernel raises a
+ * sticky status that qasr_poll_status reports as QASR_ERR_DEVICE_TIMEOUT, releases its tensor memory and
+ * ends normally.  This call enqueues one tiny kernel that runs exactly that path on purpose: it sets up
+ * as those kernels do, waits limit_us microseconds (1 .. 1 000 000) on a barrier that nothing signals,
+ * gives up and tears down.  Afterwards qasr_poll_status returns QASR_ERR_DEVICE_TIMEOUT once, and the
+ * context works as before.  (No passage of the paper: an operational aid.)  sm_100 devices only. */
+int qasr_selftest_wait_timeout(qasr_ctx* ctx, unsigned limit_us);
+
+/* Diagnostic: the int8 tensor-core throughput this GPU reaches on the instruction the convolution kernels
+ * use (tcgen05.mma kind::i8, M = 128, N = 256, K = 32), issued back to back by every SM on operands that
+ * stay in shared memory -- the denominator for "fraction of the int8 tensor peak".  Runs `kblocks` groups
+ * of four such instructions per SM (1 .. 2^20; 20 000 take about a millisecond), waits for them, and
+ * returns the device time in *ms (host pointer) and the operations done in *ops (a multiply-accumulate
+ * counts as two).  Blocking.  (No passage of the paper: a measurement aid.)  sm_100 devices only. */
+int qasr_measure_int8_tensor_peak(qasr_ctx* ctx, int kblocks, float* ms, double* ops);
+
 /* ---- single operations ------------------------------------------------------------------ */
 
 /* Depthwise K-tap convolution with per-channel requantisation (no bias, no ReLU): the
@@ -163,9 +180,11 @@ int qasr_conv(qasr_ctx* ctx, const int8_t* x, int B, int C_in, int T,
 int qasr_conv_scratch_bytes(int B, int C_in, int C_out, int T, int K, int stride, size_t* bytes);
 int qasr_set_conv_scratch(qasr_ctx* ctx, void* scratch, size_t bytes);
 
-/* One QuartzNet time-channel-separable block: depthwise K-tap conv + requant, then pointwise
- * 1x1 conv with folded-BN bias, requant and optional ReLU (qasr_dw_conv followed by qasr_conv
- * with K = 1, bit for bit).  x [B][C_in][T] -> y [B][C_out][T_out].
+/* One QuartzNet time-channel-separable block (Sec. 3 names the QuartzNet encoders; Sec. 2.2 defines
+ * the integer-only operators it is made of: integer convolution on the quantised operands, BatchNorm
+ * folded into the preceding convolution, ReLU on integers): depthwise K-tap conv + requant, then
+ * pointwise 1x1 conv with folded-BN bias, requant and optional ReLU (qasr_dw_conv followed by
+ * qasr_conv with K = 1, bit for bit).  x [B][C_in][T] -> y [B][C_out][T_out].
  * workspace: device scratch of at least qasr_tcs_block_workspace_bytes (may be NULL when that
  * is 0), 256-byte aligned; its contents are unspecified afterwards. */
 int qasr_tcs_block_workspace_bytes(int B, int C_in, int C_out, int T, int K, int stride,
@@ -195,7 +214,15 @@ int qasr_tcs_block(qasr_ctx* ctx, const int8_t* x, int B, int C_in, int T,
  *     calls whose kernels overlap on the GPU (different streams, no ordering) race on it;
  *     serialise them.
  *   - wait != 0: the call waits for the stream and also reports (and clears) the device status,
- *     i.e. QASR_ERR_RANGE for an out-of-range mult/shift entry.  wait == 0: asynchronous. */
+ *     i.e. QASR_ERR_RANGE for an out-of-range mult/shift entry.  wait == 0: asynchronous.
+ *   - Besides the array, all calls on a device share ONE status word, and it is sticky: an error
+ *     that a wait == 0 call leaves there is neither reported nor cleared until some later call
+ *     with wait != 0 on that device collects it -- possibly another caller's, on another stream
+ *     (and clearing it races with kernels of other streams still in flight).  Callers that run
+ *     asynchronously should therefore finish each batch of calls with one wait != 0 call.
+ *   - wait != 0 synchronises the stream and copies the status word back with a blocking copy, so
+ *     it cannot be used while the stream is being captured, not even after the first call.
+ *   - The call makes `device` the calling thread's current CUDA device and leaves it so. */
 #define QASR_NOALLOC_SCRATCH_BYTES (16u << 20)
 int qasr_tcs_block_noalloc(int device, void* cuda_stream,
                            const int8_t* x, int B, int C_in, int T,
@@ -203,7 +230,9 @@ int qasr_tcs_block_noalloc(int device, void* cuda_stream,
                            const int8_t* w_pw, int C_out, const int32_t* bias, int32_t max_abs_bias,
                            qasr_requant rq_pw, int relu, int8_t* y, int wait);
 
-/* Integer residual add of int8 tensors that sit at different scales:
+/* Integer residual add of int8 tensors that sit at different scales (Sec. 2.2 requires the entire
+ * inference, the residual connections of the encoders included, to run in integer arithmetic; it does
+ * not print the rule, so the per-term dyadic rescaling below is this library's reading of it):
  *   y = sat8(relu?( sum_j RS(terms[j] * mult[j], shift[j]) )),  every term rounded on its own.
  * terms: host array of n_terms (1..QASR_MAX_TERMS) device pointers [B][C][T]; mult, shift: host
  * arrays (per-tensor constants). */

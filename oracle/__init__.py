@@ -57,8 +57,6 @@ def lib():
         L.qo_rs.argtypes = [ctypes.c_int64, c_int]
         L.qo_sat8.restype = ctypes.c_int64
         L.qo_sat8.argtypes = [ctypes.c_int64]
-        L.qo_requant1.restype = ctypes.c_int8
-        L.qo_requant1.argtypes = [ctypes.c_int32, ctypes.c_int32, c_int]
         L.qo_conv1d.restype = c_int
         L.qo_conv1d.argtypes = [i8p, c_int, c_int, c_int, i8p, c_int, c_int, c_int, c_int, c_int, i32p, i32p]
         L.qo_requant.restype = c_int
@@ -99,10 +97,6 @@ def rs(v: int, c: int) -> int:
 
 def sat8(v: int) -> int:
     return int(lib().qo_sat8(int(v)))
-
-
-def requant1(acc: int, mult: int, shift: int) -> int:
-    return int(lib().qo_requant1(int(acc), int(mult), int(shift)))
 
 
 # ----------------------------------------------------------------------------- tensors

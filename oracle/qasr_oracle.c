@@ -73,11 +73,6 @@ int64_t qo_sat8(int64_t v) {
     return v;
 }
 
-/* one requantisation: int32 accumulator -> int8 code */
-int8_t qo_requant1(int32_t acc, int32_t mult, int shift) {
-    return (int8_t)qo_sat8(qo_rs((int64_t)acc * (int64_t)mult, shift));
-}
-
 static int out_len(int T, int K, int stride, int dilation) {
     (void)K; (void)dilation; /* "same" padding: pad = dilation*(K-1)/2 on both sides */
     return (T - 1) / stride + 1;

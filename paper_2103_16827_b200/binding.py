@@ -71,6 +71,10 @@ def lib():
     L.qasr_last_error.restype = ctypes.c_char_p
     L.qasr_poll_status.argtypes = [vp]
     L.qasr_set_option.argtypes = [vp, ci, ci]
+    L.qasr_selftest_wait_timeout.argtypes = [vp, ctypes.c_uint]
+    L.qasr_selftest_wait_timeout.restype = ci
+    L.qasr_measure_int8_tensor_peak.argtypes = [vp, ci, P(ctypes.c_float), P(ctypes.c_double)]
+    L.qasr_measure_int8_tensor_peak.restype = ci
     L.qasr_launch_count.argtypes = [vp]
     L.qasr_launch_count.restype = ctypes.c_int64
     L.qasr_dw_conv.argtypes = [vp, vp, ci, ci, ci, vp, ci, ci, ci, QasrRequant, vp]
@@ -187,6 +191,15 @@ class Context:
 
     def set_option(self, option, value):
         self._check(self._lib.qasr_set_option(self._h, int(option), int(value)))
+
+    def selftest_wait_timeout(self, limit_us=1000):
+        self._check(self._lib.qasr_selftest_wait_timeout(self._h, int(limit_us)))
+
+    def measure_int8_tensor_peak(self, kblocks=20000):
+        """Measured int8 tensor-core throughput in TOP/s (multiply-accumulate = 2 ops) and the device time in ms."""
+        ms, ops = ctypes.c_float(), ctypes.c_double()
+        self._check(self._lib.qasr_measure_int8_tensor_peak(self._h, int(kblocks), ctypes.byref(ms), ctypes.byref(ops)))
+        return ops.value / (ms.value * 1e-3) / 1e12, ms.value
 
     def launch_count(self):
         return int(self._lib.qasr_launch_count(self._h))

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libqasr.so")
-SOURCES = ["qasr_api.cu", "kernels_generic.cu", "fast_paths.cu", "gemm_tc.cu", "dw_dp4a.cu", "dw_tc.cu", "conv_tc.cu", "noalloc.cu"]
+SOURCES = ["qasr_api.cu", "kernels_generic.cu", "fast_paths.cu", "gemm_tc.cu", "dw_dp4a.cu", "dw_tc.cu", "conv_tc.cu", "noalloc.cu", "selftest.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC"]
 

@@ -500,9 +500,7 @@ int qasr_launch_conv_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
     p.n_items = a.B * p.tiles_t * p.m_groups;
     p.bias = a.bias; p.mult = a.mult; p.shift = a.shift; p.y = a.y; p.y32 = a.y_int32; p.relu = a.relu;
     p.terms = a.terms;
-    p.terms_fast = 1;
-    for (int j = 0; j < a.terms.n; ++j)
-        if (a.terms.mult[j] >= (1 << 23) || a.terms.shift[j] > 30) p.terms_fast = 0;
+    p.terms_fast = qasr_terms_fit_int32(a.terms) ? 1 : 0;
     p.status = ctx->d_status;
 
     for (int k = 0; k < a.K; ++k) {

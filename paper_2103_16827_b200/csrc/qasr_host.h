@@ -104,6 +104,18 @@ inline double qasr_conv_bytes(const QasrConvArgs& a) {
            (double)a.C_out * a.C_in * a.K + 9.0 * a.C_out;
 }
 
+// True if the residual stage of an epilogue can be carried in 32-bit arithmetic without changing a bit:
+// every product q * mult + 2^(shift-1) with |q| <= 128 fits int32 (mult < 2^23, shift <= 30), and so does
+// the sum of the rescaled terms, each of which is at most ((128 * mult) >> shift) + 1 in magnitude.
+inline bool qasr_terms_fit_int32(const QasrTerms& t) {
+    long long sum = 0;
+    for (int j = 0; j < t.n; ++j) {
+        if (t.mult[j] < 0 || t.mult[j] >= (1 << 23) || t.shift[j] < 1 || t.shift[j] > 30) return false;
+        sum += ((128LL * t.mult[j]) >> t.shift[j]) + 1;
+    }
+    return sum < (1LL << 31);
+}
+
 // Launches a kernel whose prologue may overlap the tail of the previous kernel in the stream
 // (programmatic dependent launch); the kernel itself must execute griddepcontrol.wait before it
 // touches anything an earlier kernel wrote or still reads.

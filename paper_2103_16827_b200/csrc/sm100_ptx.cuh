@@ -40,12 +40,13 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Bounded wait: gives up after a fixed number of polls (well under two seconds), raises the
-// sticky device status and the CTA-wide abort flag, and returns false. Callers then leave
+// Bounded wait: gives up after `limit_ns` of wall time (two seconds unless the caller says otherwise),
+// raises the sticky device status and the CTA-wide abort flag, and returns false. Callers then leave
 // their loops and fall through to the common teardown.
 // Each poll is a try_wait that may suspend the thread for up to about a microsecond, so a waiting
 // warp costs few issue slots.
 constexpr uint32_t kWaitPollsHardCap = 1u << 30;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 #ifndef QASR_WAIT_HINT_NS
 #define QASR_WAIT_HINT_NS 1000u
 #endif
@@ -61,10 +62,10 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          unsigned* status) {
+                                          unsigned* status, unsigned long long limit_ns = kWaitLimitNs) {
     if (mbar_test(bar, parity)) return true;
-    // Bound: two seconds of wall time (checked every 64 polls), with a hard cap on the poll count
-    // that cannot be reached sooner than that.
+    // Bound: limit_ns of wall time (checked every 64 polls), with a hard cap on the poll count
+    // that the default limit cannot reach sooner than that.
     unsigned long long t_start = 0;
     for (uint32_t it = 0; it < kWaitPollsHardCap; ++it) {
         if (mbar_try(bar, parity)) return true;
@@ -74,7 +75,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             unsigned long long now;
             asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
             if (t_start == 0) t_start = now;
-            if (now - t_start > 2000000000ull) break;
+            if (now - t_start > limit_ns) break;
         }
     }
     *abort_flag = 1;

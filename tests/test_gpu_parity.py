@@ -250,20 +250,100 @@ def test_conv_without_bias_and_extreme_inputs(ctx):
     assert_same(got32, acc, "extreme int32")
 
 
-@pytest.mark.parametrize("mult,shift", [(1, 1), ((1 << 31) - 1, 62), ((1 << 31) - 1, 31), (12345, 1), (1 << 30, 40), (0, 5)])
-def test_requant_constant_corners(ctx, mult, shift):
-    """Identity 1x1 weights expose the requantisation alone over the whole int8 input range."""
-    C = 16
+CORNER_RQ = [(1, 1), ((1 << 31) - 1, 62), ((1 << 31) - 1, 31), (12345, 1), (1 << 30, 40), (0, 5), (1 << 14, 32), (3, 33)]
+
+
+def _profiled(q, ctx, fn):
+    """Runs fn() in profile mode and returns (result, names of the kernels it launched)."""
+    ctx.set_option(q.OPT_PROFILE, 1)
+    ctx.profile_read()
+    out = fn()
+    kernels = [e["kernel"] for e in ctx.profile_read()]
+    ctx.set_option(q.OPT_PROFILE, 0)
+    return out, kernels
+
+
+@pytest.mark.parametrize("C,kernel", [(16, "conv_generic"), (64, "gemm_i8_tc"), (128, "gemm_i8_tc")])
+@pytest.mark.parametrize("rq", CORNER_RQ + ["mixed"])
+def test_requant_constant_corners(q, ctx, C, kernel, rq):
+    """Identity 1x1 weights expose the requantisation alone over the whole int8 input range, at the corners of
+    the range the header promises (0 <= mult < 2^31, 1 <= shift <= 62): multipliers without head-room (the
+    64-bit branch of the tensor-core epilogue), shifts below, at and above 32, and a mix of all of them across
+    the channels of one warp.  C = 64 and 128 run on the tensor-core GEMM (both pipeline block widths)."""
     x = np.tile(np.arange(-128, 128, dtype=np.int64).astype(np.int8), (1, C, 1))
     w = (np.eye(C, dtype=np.int8) * 127)[:, :, None]
     bias = (np.arange(C, dtype=np.int64) * 1000003 % 200001 - 100000).astype(np.int32)
-    m = np.full(C, mult, np.int32)
-    s = np.full(C, shift, np.uint8)
+    if rq == "mixed":
+        m = np.array([CORNER_RQ[i % len(CORNER_RQ)][0] for i in range(C)], np.int32)
+        s = np.array([CORNER_RQ[i % len(CORNER_RQ)][1] for i in range(C)], np.uint8)
+    else:
+        m = np.full(C, rq[0], np.int32)
+        s = np.full(C, rq[1], np.uint8)
     acc = oracle.conv1d(x, w, bias)
     for relu in (False, True):
         want = oracle.requant(acc, m, s, relu=relu)
-        got = ctx.conv(dev(x), dev(w), dev(bias), 100000, dev(m), dev(s), relu)
+        got, kernels = _profiled(q, ctx, lambda: ctx.conv(dev(x), dev(w), dev(bias), 100000, dev(m), dev(s), relu))
         assert_same(got, want, "requant corners")
+        assert kernels == [kernel], kernels
+
+
+def test_dw_requant_constant_corners_on_tensor_cores(q, ctx):
+    """The same corners on the tensor-core depthwise kernel: one channel (= one work item) per constant pair,
+    so every branch of its requantiser runs (shift 32 after normalisation, above 32, and the 64-bit form)."""
+    rng = np.random.default_rng(77)
+    B, T, K = 8, 256, 33
+    C = 2 * len(CORNER_RQ)
+    x = rng.integers(-128, 128, size=(B, C, T)).astype(np.int8)
+    w = rng.integers(-127, 128, size=(C, K)).astype(np.int8)
+    w[1::2] = 0
+    w[1::2, K // 2] = 1                            # odd channels: identity taps, the accumulator is the input
+    m = np.array([CORNER_RQ[i // 2][0] for i in range(C)], np.int32)
+    s = np.array([CORNER_RQ[i // 2][1] for i in range(C)], np.uint8)
+    want = oracle.requant(oracle.conv1d(x, w, None, 1, 1, depthwise=True), m, s)
+    got, kernels = _profiled(q, ctx, lambda: ctx.dw_conv(dev(x), dev(w), 1, 1, dev(m), dev(s)))
+    assert_same(got, want, "dw corners")
+    assert kernels == ["dw_conv_tc"], kernels
+    assert len(np.unique(want)) > 100
+
+
+WIDE_TERMS = {
+    "mult_2^23": ([1 << 23, 20000], [23, 15]),                     # a multiplier the 32-bit rescale cannot take
+    "shift_38": ([23170, (1 << 31) - 1], [15, 38]),                # a shift above 30
+    "sum_overflows_int32": ([(1 << 23) - 1] * 5, [1] * 5),         # every term fits 32 bits, their sum does not
+    "near_the_32bit_limit": ([1 << 22] * 3, [1, 1, 1]),            # the largest sum the 32-bit path still takes
+    "twelve_terms": ([20000 + 100 * j for j in range(12)], [15 + j % 3 for j in range(12)]),
+}
+
+
+@pytest.mark.parametrize("name", sorted(WIDE_TERMS))
+@pytest.mark.parametrize("K", [1, 5])
+def test_residual_epilogue_with_wide_term_constants(q, ctx, name, K):
+    """Residual terms whose constants leave the 32-bit fast path of the tensor-core epilogue (and one set that
+    sits just inside it), through the pointwise GEMM (K = 1) and the K-tap implicit GEMM (K = 5)."""
+    tm, ts = WIDE_TERMS[name]
+    tm, ts = np.array(tm, np.int32), np.array(ts, np.uint8)
+    n = len(tm)
+    rng = np.random.default_rng(n * 10 + K)
+    B, Ci, Co, T = 2, 128, 160, 208
+    x = rng.integers(-128, 128, size=(B, Ci, T)).astype(np.int8)
+    w = rng.integers(-127, 128, size=(Co, Ci, K)).astype(np.int8)
+    bias = rng.integers(-4096, 4097, size=Co).astype(np.int32)
+    sh = int(np.ceil(np.log2(np.sqrt(Ci * K) * 73 * 74 * 2 ** 14.5 / 40)))
+    m, s = rand_rq(rng, Co, sh - 1, sh + 1)
+    res = [rng.integers(-128, 128, size=(B, Co, T)).astype(np.int8) for _ in range(n - 1)]
+    for r in res:
+        r[0, :, :8] = 127                      # the extremes, where a 32-bit sum would wrap
+        r[1, :, :8] = -128
+    a = oracle.requant(oracle.conv1d(x, w, bias, 1, 1), m, s)
+    if K > 1:
+        ctx.set_conv_scratch(torch.zeros(max(256, ctx.conv_scratch_bytes(B, Ci, Co, T, K, 1)), dtype=torch.uint8, device="cuda"))
+    for relu in (True, False):
+        want = oracle.residual_add([a] + res, tm, ts, relu=relu)
+        got, kernels = _profiled(q, ctx, lambda: ctx.conv(dev(x), dev(w), dev(bias), 4096, dev(m), dev(s), relu, 1, 1,
+                                                          terms=[None] + [dev(r) for r in res], term_mult=tm, term_shift=ts))
+        assert_same(got, want, "residual epilogue %s K=%d" % (name, K))
+        assert kernels[-1] == ("gemm_i8_tc" if K == 1 else "conv_i8_tc"), kernels
+    ctx.set_conv_scratch(None)
 
 
 # ------------------------------------------------------------------ TCS block (config 0)
@@ -410,16 +490,48 @@ def test_encoder_forward_host_buffers(q, ctx):
     assert np.max(np.abs(lf.numpy() - wf)) <= 1e-6
 
 
-def test_config2_full_batch_sampled_utterances(q, ctx):
-    """QuartzNet-15x5 shape at B=32, T=1600 in the benchmark's launch configuration; the oracle
-    computes utterances 0 and 31 on their own (utterances are independent)."""
+def test_config2_full_batch_every_utterance(q, ctx):
+    """QuartzNet-15x5 shape at B=32, T=1600 in the benchmark's launch configuration (ping-pong buffers, graph
+    replay): the logits of all 32 utterances against the oracle."""
     model, x = workloads.config(2, variant="live")
-    gq, gf, _, _ = run_encoder(q, ctx, model, x)
-    pick = [0, 31]
-    wq, wf, _ = oracle.encoder_forward(model, x[pick], keep=False)
-    assert_same(gq[pick], wq, "config 2 logits_q (utterances 0, 31)")
-    assert np.max(np.abs(gf[pick] - wf)) <= 1e-6
+    gq, gf, _, keep = run_encoder(q, ctx, model, x)
+    wq, wf, _ = oracle.encoder_forward(model, x, keep=False)
+    assert_same(gq, wq, "config 2 logits_q (all utterances)")
+    assert np.max(np.abs(gf - wf)) <= 1e-6
     assert np.std(wq.astype(np.float64)) > 100
+    # the replayed graph gives the same bits
+    dm, ws = keep
+    lq = torch.zeros_like(torch.from_numpy(wq)).cuda()
+    lf = torch.zeros_like(torch.from_numpy(wf)).cuda()
+    xd = dev(x)
+    for _ in range(2):
+        lq.zero_()
+        ctx.encoder_forward(dm, xd, ws, lq, lf)
+    ctx.poll_status()
+    assert_same(lq, wq, "config 2 logits_q after graph replay")
+
+
+def test_config2_full_batch_every_layer_of_middle_utterances(q, ctx):
+    """The same workload with a buffer of its own for every layer (about 2 GB of workspace): every
+    intermediate tensor of utterances 13 and 22 -- middle work items of every kernel -- against the oracle."""
+    model, x = workloads.config(2, variant="live", unique_bufs=True)
+    pick = [13, 22]
+    wq, wf, trace = oracle.encoder_forward(model, x[pick])
+    dm = q.DeviceModel(model, 0)
+    B, _, T = x.shape
+    ws = torch.zeros(ctx.encoder_workspace_bytes(dm, B, T), dtype=torch.uint8, device="cuda")
+    last = model["layers"][-1]
+    lq = torch.zeros((B, last["C_out"], wq.shape[2]), dtype=torch.int32, device="cuda")
+    lf = torch.zeros(lq.shape, dtype=torch.float32, device="cuda")
+    ctx.encoder_forward(dm, dev(x), ws, lq, lf)
+    ctx.poll_status()
+    idx = torch.tensor(pick, device="cuda")
+    for L, o in zip(model["layers"][:-1], trace[:-1]):
+        off, C, Tl = ctx.encoder_buffer_info(dm, B, T, L["out"])
+        got = ws[off:off + B * C * Tl].view(torch.int8).reshape(B, C, Tl)[idx].cpu().numpy()
+        assert_same(got, o["y"], "config 2 layer " + L["name"])
+    assert_same(lq[idx].cpu().numpy(), wq, "config 2 logits_q (utterances 13, 22)")
+    assert np.max(np.abs(lf[idx].cpu().numpy() - wf)) <= 1e-6
 
 
 # ------------------------------------------------------------------ Jasper / Conformer shapes
@@ -477,10 +589,10 @@ def test_small_conformer_every_layer(q, ctx, variant):
 
 def test_config4_conformer_full_batch_sampled_utterances(q, ctx):
     model, x = workloads.config(4, variant="live")
-    pick = [0, 15]
+    pick = [0, 6, 9, 15]
     wq, wf, _ = oracle.encoder_forward(model, x[pick], keep=False)
     gq, gf, _, _ = run_encoder_T(q, ctx, model, x, wq.shape[2])
-    assert_same(gq[pick], wq, "config 4 logits_q (utterances 0, 15)")
+    assert_same(gq[pick], wq, "config 4 logits_q (utterances 0, 6, 9, 15)")
     assert np.max(np.abs(gf[pick] - wf)) <= 1e-6
     assert np.std(wq.astype(np.float64)) > 100
 
@@ -521,13 +633,13 @@ def test_static_weights_option_reuses_regrouped_weights(q, ctx):
     ctx.set_option(q.OPT_STATIC_WEIGHTS, 0)
 
 
-def test_config3_jasper_full_batch_sampled_utterance(q, ctx):
-    """JasperDR-10x5 shape at B=16, T=1600; the oracle computes utterance 5 on its own."""
+def test_config3_jasper_full_batch_sampled_utterances(q, ctx):
+    """JasperDR-10x5 shape at B=16, T=1600; the oracle computes utterances 0, 7 and 15 on their own."""
     model, x = workloads.config(3, variant="live")
-    pick = [5]
+    pick = [0, 7, 15]
     gq, gf, _, _ = run_encoder_T(q, ctx, model, x, 800)
     wq, wf, _ = oracle.encoder_forward(model, x[pick], keep=False)
-    assert_same(gq[pick], wq, "config 3 logits_q (utterance 5)")
+    assert_same(gq[pick], wq, "config 3 logits_q (utterances 0, 7, 15)")
     assert np.max(np.abs(gf[pick] - wf)) <= 1e-6
     assert np.std(wq.astype(np.float64)) > 100
 
@@ -666,6 +778,37 @@ def test_conv_with_too_little_scratch_falls_back_to_the_generic_kernel(q, ctx):
     ctx.set_conv_scratch(None)
     assert_same(got, oracle.requant(oracle.conv1d(x, w, None, 1, 1), m, s), "conv, scratch too small")
     assert kernels == ["conv_generic"], kernels
+
+
+def test_bounded_device_wait_expires_into_a_status_and_the_context_stays_usable(q, ctx):
+    """The failure-detection path of the tensor-core kernels, taken on purpose by the library's self-test
+    kernel (a wait on a barrier that nothing signals, limit 1 ms): the wait gives up, qasr_poll_status reports
+    QASR_ERR_DEVICE_TIMEOUT once, tensor memory was released (the next tensor-core kernels run and are
+    bit-exact), and nothing hangs."""
+    import time
+    t0 = time.perf_counter()
+    ctx.selftest_wait_timeout(1000)
+    with pytest.raises(q.QasrError) as e:
+        ctx.poll_status()
+    assert e.value.code == -8
+    assert time.perf_counter() - t0 < 5.0
+    ctx.poll_status()                       # sticky status was cleared by the read
+    rng = np.random.default_rng(4)
+    B, Ci, Co, T = 8, 128, 128, 256
+    x = rng.integers(-128, 128, size=(B, Ci, T)).astype(np.int8)
+    w = rng.integers(-127, 128, size=(Co, Ci, 1)).astype(np.int8)
+    wd = rng.integers(-127, 128, size=(Ci, 33)).astype(np.int8)
+    m, s = rand_rq(rng, Co, 25, 27)
+    md, sd = rand_rq(rng, Ci, 20, 22)
+    got, kernels = _profiled(q, ctx, lambda: ctx.conv(dev(x), dev(w), None, 0, dev(m), dev(s), True))
+    assert kernels == ["gemm_i8_tc"], kernels
+    assert_same(got, oracle.requant(oracle.conv1d(x, w, None), m, s, relu=True), "conv after a timed-out wait")
+    got, kernels = _profiled(q, ctx, lambda: ctx.dw_conv(dev(x), dev(wd), 1, 1, dev(md), dev(sd)))
+    assert kernels == ["dw_conv_tc"], kernels
+    assert_same(got, oracle.requant(oracle.conv1d(x, wd, None, 1, 1, depthwise=True), md, sd), "dw after a timed-out wait")
+    with pytest.raises(q.QasrError) as e:
+        ctx.selftest_wait_timeout(0)
+    assert e.value.code == -2
 
 
 def test_out_of_range_device_constants_raise_status_not_fault(q, ctx):

@@ -455,6 +455,85 @@ def test_live_variant_keeps_tensors_alive_and_literal_collapses():
 
 
 # ------------------------------------------------------------------ integer GLU gate (paper parity unpinned)
+def _read_gate(q_c):
+    """The gate value sig(g) of oracle.glu for every int8 g, read out exactly through the output alone.
+    With a = 1 and (mult, shift) = (ceil(2^30 / theta), 31) the output RS(sig * mult, 31) is >= 1 exactly
+    when sig >= theta (theta <= 2^15, sig an integer), so each call is an exact comparator; every g sits
+    in a channel of its own and a bisection over theta finds its sig.  Nothing of the gate's formula is
+    used here, only the rounding shift that the tests above pin."""
+    g = np.arange(-128, 128, dtype=np.int64)
+    q = g.astype(np.int8).reshape(1, 256, 1)
+    a = np.ones_like(q)
+    lo = np.zeros(256, np.int64)              # sig >= lo always holds (sig >= 0)
+    hi = np.full(256, (1 << 15) + 1, np.int64)    # sig < hi
+    while np.any(hi - lo > 1):
+        theta = np.maximum((lo + hi) // 2, 1)
+        mult = (-(-(1 << 30) // theta)).astype(np.int32)          # ceil(2^30 / theta)
+        y = oracle.glu(a, q, q_c, mult, np.full(256, 31, np.uint8))[0, :, 0]
+        ge = y >= 1
+        lo = np.where(ge, theta, lo)
+        hi = np.where(ge, hi, theta)
+    return g, lo
+
+
+@pytest.mark.parametrize("q_c", [1, 2, 7, 80, 117, 127, 128])
+def test_glu_gate_is_the_piecewise_quadratic_its_definition_states(q_c):
+    """Exact pins of the library's own gate (the paper prints no coefficients): anchor values, saturation,
+    point symmetry about (0, q_c^2), monotonicity, and constant second differences -2 on (0, q_c) and +2 on
+    (-q_c, 0).  A quadratic is fixed by two anchors and its second difference, so these leave no freedom:
+    an off-by-one in the clamp, in p or in a sign fails one of them."""
+    g, sig = _read_gate(q_c)
+    at = dict(zip(g.tolist(), sig.tolist()))
+    full = 2 * q_c * q_c
+    assert at[0] == q_c * q_c
+    for v in range(-128, 128):
+        if v >= q_c:
+            assert at[v] == full, v
+        if v <= -q_c:
+            assert at[v] == 0, v
+        if -127 <= v <= 127:
+            assert at[v] + at[-v] == full, v              # point symmetry
+        if v > -128:
+            assert at[v] >= at[v - 1], v                  # monotone
+        if -127 <= v <= 126:
+            d2 = at[v + 1] - 2 * at[v] + at[v - 1]
+            if 0 < v < q_c:
+                assert d2 == -2, (v, d2)
+            elif -q_c < v < 0:
+                assert d2 == 2, (v, d2)
+            elif abs(v) > q_c:
+                assert d2 == 0, (v, d2)
+    # strictly increasing inside the unsaturated range
+    for v in range(max(-q_c, -127), min(q_c, 127)):
+        assert at[v + 1] > at[v], v
+
+
+def test_glu_output_is_the_rounded_product_of_value_gate_and_multiplier():
+    """y = sat8(RS(a * sig * mult, shift)) with Python integers, sig taken from the read-out table (not from
+    a formula): pins the product, the 64-bit range, the rounding and the clamp of the output stage."""
+    rng = np.random.default_rng(21)
+    for q_c in (5, 80, 128):
+        g, sig = _read_gate(q_c)
+        C, T = 12, 256
+        a = rng.integers(-128, 128, size=(2, C, T)).astype(np.int8)
+        q = rng.integers(-128, 128, size=(2, C, T)).astype(np.int8)
+        a[0, 0, :] = np.arange(-128, 128)
+        q[0, 1, :] = np.arange(-128, 128)
+        mult = rng.integers(0, 1 << 31, size=C).astype(np.int32)
+        shift = rng.integers(1, 63, size=C).astype(np.uint8)
+        mult[0], shift[0] = 1, 1
+        mult[1], shift[1] = (1 << 31) - 1, 62
+        mult[2], shift[2] = (1 << 31) - 1, 20          # saturates both ways
+        mult[3], shift[3] = 0, 7
+        y = oracle.glu(a, q, q_c, mult, shift)
+        for b in range(2):
+            for c in range(C):
+                for t in range(0, T, 3):
+                    v = int(a[b, c, t]) * int(sig[int(q[b, c, t]) + 128]) * int(mult[c])
+                    want = max(-128, min(127, _rs_exact(v, int(shift[c]))))
+                    assert int(y[b, c, t]) == want, (q_c, b, c, t)
+
+
 def test_glu_gate_tracks_a_sigmoid():
     q_c = 80                       # S = 4 / q_c
     S = 4.0 / q_c
