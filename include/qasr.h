@@ -86,10 +86,9 @@ int qasr_poll_status(qasr_ctx* ctx);
 /* Options.  QASR_OPT_GRAPH (default 1): qasr_encoder_forward replays a captured CUDA graph when
  * called again with identical arguments.  QASR_OPT_TENSOR_CORES (default 1): pointwise/dense
  * convolutions use the tcgen05 path when the shape allows it (0 forces the generic kernels).
- * QASR_OPT_FUSE_TCS (default 1): depthwise+pointwise run as one kernel when the shape allows it. */
+ * (Option id 3 is not in use.) */
 #define QASR_OPT_GRAPH 1
 #define QASR_OPT_TENSOR_CORES 2
-#define QASR_OPT_FUSE_TCS 3
 /* QASR_OPT_PROFILE (default 0): every kernel is launched on its own (no graph) between two CUDA
  * events; qasr_profile_read returns one record per launch. */
 #define QASR_OPT_PROFILE 4

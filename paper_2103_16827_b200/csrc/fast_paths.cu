@@ -1,4 +1,4 @@
-// Dispatch of the vectorised depthwise kernel, the tcgen05 GEMM and the fused TCS kernel: each
+// Dispatch of the depthwise kernels and of the tcgen05 GEMM / implicit-GEMM kernels: each
 // function decides whether the shape qualifies and, if so, enqueues the fast kernel.
 #include <cstdio>
 
@@ -17,7 +17,6 @@ static inline bool al16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 int qasr_host_init(qasr_ctx* ctx) {
     if (ctx->cc_major != 10) {   // the tensor-core and TMA kernels are sm_100a code
         ctx->opt_tc = false;
-        ctx->opt_fuse = false;
         return QASR_OK;
     }
     void* fn = nullptr;
@@ -59,9 +58,4 @@ int qasr_try_conv_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
         return rc == QASR_OK ? 1 : rc;
     }
     return qasr_launch_conv_tc(ctx, a);         // K taps / stride / odd channel counts: implicit GEMM, needs scratch
-}
-
-int qasr_try_tcs_fused(qasr_ctx* ctx, const QasrDwArgs& d, const QasrConvArgs& p) {
-    (void)ctx; (void)d; (void)p;
-    return 0;
 }

@@ -53,6 +53,7 @@ struct GemmParams {
     int out_bytes;                 // bytes of the output staging area (one block per epilogue warp)
     int stage_w;                   // bytes per staged row of the wider warps (16 * ceil(chunks / EPI_PARTS))
     int epi_parts;                 // epilogue warps per quarter (the kernel's template parameter)
+    int acc_sleep_ns;              // back-off of the MMA warp between polls for a free accumulator buffer
     const int32_t* bias;
     const int32_t* mult;
     const uint8_t* shift;
@@ -71,6 +72,7 @@ struct SharedTail {
     uint64_t accfull[2], accempty[2];
     uint32_t tmem_base;
     volatile int abort_flag;
+    volatile int epi_go[2];        // per accumulator buffer: the polling epilogue warp saw it complete (0: it gave up)
 };
 
 __device__ __forceinline__ void item_coords(const GemmParams& p, int item, int& b, int& t0, int& m_lo, int& m_hi) {
@@ -121,7 +123,7 @@ __device__ __forceinline__ void epilogue_batch(const Params& p, const EpiThread&
     }
 }
 
-template <int BK, int EPI_PARTS, int BATCH>
+template <int BK, int EPI_PARTS, int BATCH, bool POLLER>
 __global__ void __launch_bounds__(threads_for(EPI_PARTS), 1)
 gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                   const __grid_constant__ CUtensorMap tmXl,
@@ -267,7 +269,8 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                 const int rot_k = (blockIdx.x / mc) % KB;
                 for (int mi = 0; mi < mc && ok; ++mi, ++acount) {
                     const int a = acount & 1u;
-                    ok = ptx::mbar_wait(ptx::smem_u32(&sh->accempty[a]), ((acount >> 1) & 1u) ^ 1u, abort_flag, p.status);
+                    ok = ptx::mbar_wait(ptx::smem_u32(&sh->accempty[a]), ((acount >> 1) & 1u) ^ 1u, abort_flag, p.status,
+                                        ptx::kWaitLimitNs, (unsigned)p.acc_sleep_ns);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     ptx::tc_fence_after();
@@ -346,8 +349,20 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                     __syncwarp();
                 }
-                ok = ptx::mbar_wait(ptx::smem_u32(&sh->accfull[a]), (acount >> 1) & 1u, abort_flag, p.status);
-                ok = __all_sync(0xffffffffu, ok);
+                // One epilogue warp polls the barrier; the others sleep in a hardware barrier until it has seen the
+                // accumulator, so that waiting warps take no issue slots from the MMA warp and from one another.
+                // The polling warp always arrives (its wait is bounded) and passes its verdict on through shared memory.
+                if (POLLER) {
+                    if (warp == 2) {
+                        const bool seen = ptx::mbar_wait(ptx::smem_u32(&sh->accfull[a]), (acount >> 1) & 1u, abort_flag, p.status);
+                        if (lane == 0) sh->epi_go[a] = seen ? 1 : 0;
+                    }
+                    asm volatile("bar.sync 1, %0;" ::"n"(32 * EPI_WARPS) : "memory");
+                    ok = sh->epi_go[a] != 0;
+                } else {
+                    ok = ptx::mbar_wait(ptx::smem_u32(&sh->accfull[a]), (acount >> 1) & 1u, abort_flag, p.status);
+                    ok = __all_sync(0xffffffffu, ok);
+                }
                 if (!ok) break;
                 ptx::tc_fence_after();
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + a * ACC_STRIDE;
@@ -431,22 +446,22 @@ static const size_t kSmemLimit = 227 * 1024;
 // The instantiations the host can pick from: (epilogue warps per quarter, chunks per TMEM load batch).
 typedef void (*GemmKernel)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap,
                            const qasr::tc::GemmParams);
-struct GemmVariant { int parts, batch; GemmKernel k64, k128; };
-#define QASR_GEMM_VARIANT(P, Bt) {P, Bt, qasr::tc::gemm_i8_tc_kernel<64, P, Bt>, qasr::tc::gemm_i8_tc_kernel<128, P, Bt>}
+struct GemmVariant { int parts, batch, poller; GemmKernel k64, k128; };
+#define QASR_GEMM_VARIANT(P, Bt, Po) {P, Bt, Po, qasr::tc::gemm_i8_tc_kernel<64, P, Bt, Po != 0>, qasr::tc::gemm_i8_tc_kernel<128, P, Bt, Po != 0>}
 static const GemmVariant kGemmVariants[] = {
-    QASR_GEMM_VARIANT(4, 1), QASR_GEMM_VARIANT(4, 2), QASR_GEMM_VARIANT(4, 4),
-    QASR_GEMM_VARIANT(3, 4), QASR_GEMM_VARIANT(3, 2), QASR_GEMM_VARIANT(2, 4), QASR_GEMM_VARIANT(2, 2),
+    QASR_GEMM_VARIANT(4, 1, 0), QASR_GEMM_VARIANT(4, 1, 1), QASR_GEMM_VARIANT(4, 2, 1),
+    QASR_GEMM_VARIANT(3, 2, 0), QASR_GEMM_VARIANT(3, 2, 1), QASR_GEMM_VARIANT(3, 4, 1), QASR_GEMM_VARIANT(2, 2, 1), QASR_GEMM_VARIANT(2, 4, 1),
 };
 static const int kNumGemmVariants = (int)(sizeof(kGemmVariants) / sizeof(kGemmVariants[0]));
 
 static int gemm_variant_index() {
     static int chosen = -1;
     if (chosen >= 0) return chosen;
-    int parts = 4, batch = 1;
-    if (const char* ev = getenv("QASR_GEMM_EPI")) sscanf(ev, "%d,%d", &parts, &batch);
+    int parts = 4, batch = 1, poller = 0;
+    if (const char* ev = getenv("QASR_GEMM_EPI")) sscanf(ev, "%d,%d,%d", &parts, &batch, &poller);
     chosen = 0;
     for (int i = 0; i < kNumGemmVariants; ++i)
-        if (kGemmVariants[i].parts == parts && kGemmVariants[i].batch == batch) chosen = i;
+        if (kGemmVariants[i].parts == parts && kGemmVariants[i].batch == batch && kGemmVariants[i].poller == poller) chosen = i;
     return chosen;
 }
 
@@ -497,6 +512,8 @@ int qasr_launch_gemm_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
     GemmParams p;
     memset(&p, 0, sizeof(p));
     p.epi_parts = EPI_PARTS;
+    p.acc_sleep_ns = 20;
+    if (const char* ev = getenv("QASR_GEMM_ACC_SLEEP")) p.acc_sleep_ns = atoi(ev);
     p.B = a.B; p.C_in = a.C_in; p.C_out = a.C_out; p.T = a.T_out;
     p.m_tiles = (a.C_out + BM - 1) / BM;
     choose_tiles(ctx->sm_count, a.B, a.T_out, p.m_tiles, a.C_in <= 512 ? 2 : 1, p);

@@ -122,7 +122,6 @@ extern "C" int qasr_tcs_block_noalloc(int device, void* cuda_stream,
     ctx.cc_major = d->cc_major;
     ctx.encode_tiled = d->encode_tiled;
     ctx.opt_tc = d->tc_ok;
-    ctx.opt_fuse = false;
     ctx.opt_graph = false;
 
     int8_t* h = (int8_t*)d->scratch;

@@ -114,7 +114,6 @@ extern "C" int qasr_set_option(qasr_ctx* ctx, int option, int value) {
     switch (option) {
         case QASR_OPT_GRAPH: ctx->opt_graph = value != 0; break;
         case QASR_OPT_TENSOR_CORES: ctx->opt_tc = value != 0; break;
-        case QASR_OPT_FUSE_TCS: ctx->opt_fuse = value != 0; break;
         case QASR_OPT_PROFILE: ctx->profiling = value != 0; break;
         case QASR_OPT_STATIC_WEIGHTS:
             ctx->opt_static_w = value != 0;
@@ -156,7 +155,6 @@ extern "C" const char* qasr_kernel_name(int kernel) {
         case QASR_K_DEQUANT: return "dequant";
         case QASR_K_DW_DP4A: return "dw_conv_dp4a";
         case QASR_K_GEMM_TC: return "gemm_i8_tc";
-        case QASR_K_TCS_FUSED: return "tcs_fused";
         case QASR_K_CONV_TC: return "conv_i8_tc";
         case QASR_K_GLU: return "glu";
         case QASR_K_CONV_PREP: return "conv_tc_prepare";
@@ -247,9 +245,6 @@ static QasrPrefetch dw_constants(const int8_t* w, const int32_t* mult, const uin
 }
 
 static int run_tcs(qasr_ctx* ctx, const QasrDwArgs& d, QasrConvArgs p, void* scratch) {
-    int used = qasr_try_tcs_fused(ctx, d, p);
-    if (used < 0) return used;
-    if (used) return QASR_OK;
     QasrDwArgs d2 = d;
     d2.y = (int8_t*)scratch;
     p.x = (const int8_t*)scratch;
@@ -363,7 +358,7 @@ extern "C" int qasr_tcs_block_workspace_bytes(int B, int C_in, int C_out, int T,
         (stride != 1 && stride != 2) || (dilation != 1 && dilation != 2))
         return QASR_ERR_SHAPE;
     const size_t t_out = (size_t)(T - 1) / stride + 1;
-    *bytes = ((size_t)B * C_in * t_out + 255) / 256 * 256;  // the depthwise output when not fused
+    *bytes = ((size_t)B * C_in * t_out + 255) / 256 * 256;  // the depthwise output
     return QASR_OK;
 }
 

@@ -20,7 +20,7 @@ struct QasrPlanKey {
 // kernel ids reported by the profiler
 enum QasrKernelId {
     QASR_K_DW_GENERIC = 1, QASR_K_CONV_GENERIC = 2, QASR_K_RESIDUAL_ADD = 3, QASR_K_DEQUANT = 4,
-    QASR_K_DW_DP4A = 5, QASR_K_GEMM_TC = 6, QASR_K_TCS_FUSED = 7, QASR_K_CONV_TC = 8, QASR_K_GLU = 9,
+    QASR_K_DW_DP4A = 5, QASR_K_GEMM_TC = 6, QASR_K_CONV_TC = 8, QASR_K_GLU = 9,
     QASR_K_DW_TC = 10, QASR_K_CONV_PREP = 11
 };
 
@@ -36,7 +36,7 @@ struct qasr_ctx {
     unsigned* d_status = nullptr;
     int sm_count = 148;
     int cc_major = 0;
-    bool opt_graph = true, opt_tc = true, opt_fuse = true, opt_pdl = true, opt_static_w = false;
+    bool opt_graph = true, opt_tc = true, opt_pdl = true, opt_static_w = false;
     int64_t launches = 0;
     char err[512] = {0};
     // cached CUDA graph of the last qasr_encoder_forward call
@@ -146,4 +146,3 @@ size_t qasr_conv_tc_input_bytes(int B, int C_in, int T, int stride);
 size_t qasr_conv_tc_weight_bytes(int C_in, int C_out, int K);
 // True if the pointwise GEMM kernel takes this shape (then no scratch is needed).
 bool qasr_conv_shape_fits_gemm(int C_in, int K, int stride, int dilation, int T_out);
-int qasr_try_tcs_fused(qasr_ctx* ctx, const QasrDwArgs& d, const QasrConvArgs& p);

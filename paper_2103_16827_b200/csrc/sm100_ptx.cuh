@@ -62,14 +62,15 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          unsigned* status, unsigned long long limit_ns = kWaitLimitNs) {
+                                          unsigned* status, unsigned long long limit_ns = kWaitLimitNs,
+                                          unsigned sleep_ns = 20) {
     if (mbar_test(bar, parity)) return true;
     // Bound: limit_ns of wall time (checked every 64 polls), with a hard cap on the poll count
     // that the default limit cannot reach sooner than that.
     unsigned long long t_start = 0;
     for (uint32_t it = 0; it < kWaitPollsHardCap; ++it) {
         if (mbar_try(bar, parity)) return true;
-        __nanosleep(20);      // a waiting warp leaves its issue slots to the warps that work
+        __nanosleep(sleep_ns);      // a waiting warp leaves its issue slots to the warps that work
         if ((it & 63u) == 63u) {
             if (*abort_flag) return false;
             unsigned long long now;

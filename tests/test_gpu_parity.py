@@ -469,7 +469,6 @@ def test_config1_pingpong_buffers_and_graph_replay(q, ctx):
     # and with every fast path switched off the bits are the same
     ctx.set_option(q.OPT_GRAPH, 0)
     ctx.set_option(q.OPT_TENSOR_CORES, 0)
-    ctx.set_option(q.OPT_FUSE_TCS, 0)
     lq.zero_()
     ctx.encoder_forward(dm, xd, ws, lq, lf)
     assert_same(lq, wq, "logits_q generic kernels")
