@@ -18,7 +18,6 @@
 // also clips the ragged edges (frames >= T, channels >= C_out); the epilogue warps never wait for
 // one another.
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 
 #include "qasr_device.cuh"
@@ -35,11 +34,9 @@ constexpr int BM = 128;            // output channels per MMA tile (TMEM lanes)
 constexpr int MAX_W_STAGES = 8;    // weight ring: as many stages as shared memory leaves room for
 constexpr int MAX_KB = 16;         // C_in <= 1024
 static_assert(MAX_KB + MAX_W_STAGES + 2 <= 31, "the barriers are initialised by one warp, one lane each");
-// EPI_PARTS epilogue warps per 32-channel quarter split a tile's frames; a template parameter of the kernel
-// (the host picks it per shape), as is the number of 16-column chunks a warp reads from TMEM before it waits.
-constexpr int MAX_EPI_PARTS = 4;
-__host__ __device__ constexpr int epi_warps(int parts) { return 4 * parts; }
-__host__ __device__ constexpr int threads_for(int parts) { return 64 + 32 * epi_warps(parts); }
+constexpr int EPI_PARTS = 4;        // epilogue warps per 32-channel quarter (they split the frames)
+constexpr int EPI_WARPS = 4 * EPI_PARTS;
+constexpr int THREADS = 64 + 32 * EPI_WARPS;
 constexpr int ACC_STRIDE = 256;    // TMEM columns between the two accumulator buffers
 constexpr int TMEM_COLS = 512;
 
@@ -52,15 +49,13 @@ struct GemmParams {
     int w_stages;                  // depth of the weight ring (<= MAX_W_STAGES)
     int out_bytes;                 // bytes of the output staging area (one block per epilogue warp)
     int stage_w;                   // bytes per staged row of the wider warps (16 * ceil(chunks / EPI_PARTS))
-    int epi_parts;                 // epilogue warps per quarter (the kernel's template parameter)
-    int acc_sleep_ns;              // back-off of the MMA warp between polls for a free accumulator buffer
     const int32_t* bias;
     const int32_t* mult;
     const uint8_t* shift;
     int8_t* y;
     int32_t* y32;
     int relu;
-    int terms_fast;                // every residual multiplier < 2^23 and shift <= 30: 32-bit rescale is exact
+    int terms_fast;                // the residual stage fits 32-bit arithmetic bit for bit (qasr_terms_fit_int32)
     QasrTerms terms;
     unsigned* status;
     QasrPrefetch next;             // constants of the kernel that follows
@@ -72,7 +67,6 @@ struct SharedTail {
     uint64_t accfull[2], accempty[2];
     uint32_t tmem_base;
     volatile int abort_flag;
-    volatile int epi_go[2];        // per accumulator buffer: the polling epilogue warp saw it complete (0: it gave up)
 };
 
 __device__ __forceinline__ void item_coords(const GemmParams& p, int item, int& b, int& t0, int& m_lo, int& m_hi) {
@@ -85,46 +79,8 @@ __device__ __forceinline__ void item_coords(const GemmParams& p, int item, int& 
     m_hi = min(p.m_tiles, m_lo + per);
 }
 
-// One batch of NB 16-column chunks of an accumulator tile: all TMEM loads are issued before the first wait,
-// so a warp pays the load latency once per batch instead of once per chunk.
-template <int NB, class Params>
-__device__ __forceinline__ void epilogue_batch(const Params& p, const EpiThread& e, uint32_t taddr, int c0, int t0,
-                                               int mode, uint8_t* orow) {
-    uint32_t r[NB][16];
-    __syncwarp();
-#pragma unroll
-    for (int i = 0; i < NB; ++i) ptx::tmem_ld16(taddr + (c0 + i) * 16, r[i]);
-#pragma unroll
-    for (int i = 0; i < NB; ++i) ptx::tmem_ld_wait(r[i]);     // the first waits for every load above, the others pass
-#pragma unroll
-    for (int i = 0; i < NB; ++i) {
-        const int c = c0 + i;
-        if (p.y32) {
-            const int t = t0 + c * 16;
-            if (e.valid_o && t < p.T) {     // T is a multiple of 16: all-or-nothing
-                int4* dst = reinterpret_cast<int4*>(p.y32 + e.row + t);
-#pragma unroll
-                for (int v = 0; v < 4; ++v)
-                    dst[v] = make_int4((int)r[i][4 * v] + e.bias, (int)r[i][4 * v + 1] + e.bias,
-                                       (int)r[i][4 * v + 2] + e.bias, (int)r[i][4 * v + 3] + e.bias);
-            }
-            continue;
-        }
-        int4 out;
-        if (mode == 0) {
-            out = p.relu ? requant16<0, true>(r[i], e.rq) : requant16<0, false>(r[i], e.rq);
-        } else if (mode == 1) {
-            out = p.relu ? requant16<1, true>(r[i], e.rq) : requant16<1, false>(r[i], e.rq);
-        } else {
-            const int t = t0 + c * 16;
-            out = epilogue16(p, e, r[i], t, e.valid_o && t < p.T);
-        }
-        *reinterpret_cast<int4*>(orow + c * 16) = out;
-    }
-}
-
-template <int BK, int EPI_PARTS, int BATCH, bool POLLER>
-__global__ void __launch_bounds__(threads_for(EPI_PARTS), 1)
+template <int BK>
+__global__ void __launch_bounds__(THREADS, 1)
 gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                   const __grid_constant__ CUtensorMap tmXl,
                   const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmYw,
@@ -140,7 +96,6 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     uint8_t* Os = Ws + W_STAGES * W_STAGE_BYTES;                // [128 channels][BN frames] output staging
     SharedTail* sh = (SharedTail*)(Os + p.out_bytes);
 
-    constexpr int EPI_WARPS = epi_warps(EPI_PARTS);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     // one barrier (pair) per thread of warp 2, so that the set-up is not one thread's serial chain
@@ -269,8 +224,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                 const int rot_k = (blockIdx.x / mc) % KB;
                 for (int mi = 0; mi < mc && ok; ++mi, ++acount) {
                     const int a = acount & 1u;
-                    ok = ptx::mbar_wait(ptx::smem_u32(&sh->accempty[a]), ((acount >> 1) & 1u) ^ 1u, abort_flag, p.status,
-                                        ptx::kWaitLimitNs, (unsigned)p.acc_sleep_ns);
+                    ok = ptx::mbar_wait(ptx::smem_u32(&sh->accempty[a]), ((acount >> 1) & 1u) ^ 1u, abort_flag, p.status);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     ptx::tc_fence_after();
@@ -349,31 +303,39 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                     __syncwarp();
                 }
-                // One epilogue warp polls the barrier; the others sleep in a hardware barrier until it has seen the
-                // accumulator, so that waiting warps take no issue slots from the MMA warp and from one another.
-                // The polling warp always arrives (its wait is bounded) and passes its verdict on through shared memory.
-                if (POLLER) {
-                    if (warp == 2) {
-                        const bool seen = ptx::mbar_wait(ptx::smem_u32(&sh->accfull[a]), (acount >> 1) & 1u, abort_flag, p.status);
-                        if (lane == 0) sh->epi_go[a] = seen ? 1 : 0;
-                    }
-                    asm volatile("bar.sync 1, %0;" ::"n"(32 * EPI_WARPS) : "memory");
-                    ok = sh->epi_go[a] != 0;
-                } else {
-                    ok = ptx::mbar_wait(ptx::smem_u32(&sh->accfull[a]), (acount >> 1) & 1u, abort_flag, p.status);
-                    ok = __all_sync(0xffffffffu, ok);
-                }
+                ok = ptx::mbar_wait(ptx::smem_u32(&sh->accfull[a]), (acount >> 1) & 1u, abort_flag, p.status);
+                ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 ptx::tc_fence_after();
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + a * ACC_STRIDE;
                 uint8_t* orow = Ow + lane * my_w - c_lo * 16;      // chunk c lands at orow + 16 * c
 
-                for (int c0 = c_lo; c0 < c_hi; c0 += BATCH) {
-                    const int nb = min(BATCH, c_hi - c0);        // warp-uniform
-                    if (BATCH >= 4 && nb == 4) epilogue_batch<4>(p, e, taddr, c0, t0, mode, orow);
-                    else if (BATCH >= 3 && nb == 3) epilogue_batch<3>(p, e, taddr, c0, t0, mode, orow);
-                    else if (BATCH >= 2 && nb == 2) epilogue_batch<2>(p, e, taddr, c0, t0, mode, orow);
-                    else epilogue_batch<1>(p, e, taddr, c0, t0, mode, orow);
+                for (int c = c_lo; c < c_hi; ++c) {
+                    uint32_t r[16];
+                    __syncwarp();
+                    ptx::tmem_ld16(taddr + c * 16, r);
+                    ptx::tmem_ld_wait(r);
+                    if (p.y32) {
+                        const int t = t0 + c * 16;
+                        if (e.valid_o && t < p.T) {     // T is a multiple of 16: all-or-nothing
+                            int4* dst = reinterpret_cast<int4*>(p.y32 + e.row + t);
+#pragma unroll
+                            for (int v = 0; v < 4; ++v)
+                                dst[v] = make_int4((int)r[4 * v] + e.bias, (int)r[4 * v + 1] + e.bias,
+                                                   (int)r[4 * v + 2] + e.bias, (int)r[4 * v + 3] + e.bias);
+                        }
+                        continue;
+                    }
+                    int4 out;
+                    if (mode == 0) {
+                        out = p.relu ? requant16<0, true>(r, e.rq) : requant16<0, false>(r, e.rq);
+                    } else if (mode == 1) {
+                        out = p.relu ? requant16<1, true>(r, e.rq) : requant16<1, false>(r, e.rq);
+                    } else {
+                        const int t = t0 + c * 16;
+                        out = epilogue16(p, e, r, t, e.valid_o && t < p.T);
+                    }
+                    *reinterpret_cast<int4*>(orow + c * 16) = out;
                 }
                 // accumulator drained: hand the TMEM buffer back to the MMA warp
                 ptx::tc_fence_before();
@@ -443,35 +405,10 @@ bool qasr_encode_map_u8(qasr_ctx* ctx, CUtensorMap* map, const void* base, int r
 
 static const size_t kSmemLimit = 227 * 1024;
 
-// The instantiations the host can pick from: (epilogue warps per quarter, chunks per TMEM load batch).
-typedef void (*GemmKernel)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap,
-                           const qasr::tc::GemmParams);
-struct GemmVariant { int parts, batch, poller; GemmKernel k64, k128; };
-#define QASR_GEMM_VARIANT(P, Bt, Po) {P, Bt, Po, qasr::tc::gemm_i8_tc_kernel<64, P, Bt, Po != 0>, qasr::tc::gemm_i8_tc_kernel<128, P, Bt, Po != 0>}
-static const GemmVariant kGemmVariants[] = {
-    QASR_GEMM_VARIANT(4, 1, 0), QASR_GEMM_VARIANT(4, 1, 1), QASR_GEMM_VARIANT(4, 2, 1),
-    QASR_GEMM_VARIANT(3, 2, 0), QASR_GEMM_VARIANT(3, 2, 1), QASR_GEMM_VARIANT(3, 4, 1), QASR_GEMM_VARIANT(2, 2, 1), QASR_GEMM_VARIANT(2, 4, 1),
-};
-static const int kNumGemmVariants = (int)(sizeof(kGemmVariants) / sizeof(kGemmVariants[0]));
-
-static int gemm_variant_index() {
-    static int chosen = -1;
-    if (chosen >= 0) return chosen;
-    int parts = 4, batch = 1, poller = 0;
-    if (const char* ev = getenv("QASR_GEMM_EPI")) sscanf(ev, "%d,%d,%d", &parts, &batch, &poller);
-    chosen = 0;
-    for (int i = 0; i < kNumGemmVariants; ++i)
-        if (kGemmVariants[i].parts == parts && kGemmVariants[i].batch == batch && kGemmVariants[i].poller == poller) chosen = i;
-    return chosen;
-}
-
 int qasr_gemm_tc_init(qasr_ctx* ctx) {
-    cudaError_t e = cudaSuccess;
-    for (int i = 0; i < kNumGemmVariants && e == cudaSuccess; ++i) {
-        e = cudaFuncSetAttribute(kGemmVariants[i].k64, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(kGemmVariants[i].k128, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
-    }
+    cudaError_t e = cudaFuncSetAttribute(qasr::tc::gemm_i8_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(qasr::tc::gemm_i8_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
     if (e != cudaSuccess) {
         snprintf(ctx->err, sizeof(ctx->err), "cudaFuncSetAttribute(gemm_i8_tc_kernel) failed: %s", cudaGetErrorString(e));
         return QASR_ERR_CUDA;
@@ -507,13 +444,8 @@ static void choose_tiles(int sm_count, int B, int T, int m_tiles, int nc_max, qa
 // 16-byte aligned tensors.
 int qasr_launch_gemm_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
     using namespace qasr::tc;
-    const GemmVariant& var = kGemmVariants[gemm_variant_index()];
-    const int EPI_PARTS = var.parts, EPI_WARPS = epi_warps(var.parts), THREADS = threads_for(var.parts);
     GemmParams p;
     memset(&p, 0, sizeof(p));
-    p.epi_parts = EPI_PARTS;
-    p.acc_sleep_ns = 20;
-    if (const char* ev = getenv("QASR_GEMM_ACC_SLEEP")) p.acc_sleep_ns = atoi(ev);
     p.B = a.B; p.C_in = a.C_in; p.C_out = a.C_out; p.T = a.T_out;
     p.m_tiles = (a.C_out + BM - 1) / BM;
     choose_tiles(ctx->sm_count, a.B, a.T_out, p.m_tiles, a.C_in <= 512 ? 2 : 1, p);
@@ -567,8 +499,8 @@ int qasr_launch_gemm_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
     const int grid = p.n_items < ctx->sm_count ? p.n_items : ctx->sm_count;
     QasrLaunchScope ls(ctx, QASR_K_GEMM_TC, qasr_conv_macs(a), qasr_conv_bytes(a));
     cudaError_t e = BK == 128
-        ? qasr_launch_overlapped(ctx, var.k128, dim3(grid), dim3(THREADS), smem, tmW, tmX, tmXl, tmY, tmYw, p)
-        : qasr_launch_overlapped(ctx, var.k64, dim3(grid), dim3(THREADS), smem, tmW, tmX, tmXl, tmY, tmYw, p);
+        ? qasr_launch_overlapped(ctx, gemm_i8_tc_kernel<128>, dim3(grid), dim3(THREADS), smem, tmW, tmX, tmXl, tmY, tmYw, p)
+        : qasr_launch_overlapped(ctx, gemm_i8_tc_kernel<64>, dim3(grid), dim3(THREADS), smem, tmW, tmX, tmXl, tmY, tmYw, p);
     if (e != cudaSuccess) {
         snprintf(ctx->err, sizeof(ctx->err), "gemm_i8_tc_kernel launch failed: %s", cudaGetErrorString(e));
         return QASR_ERR_CUDA;
