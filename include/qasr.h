@@ -98,6 +98,13 @@ int qasr_poll_status(qasr_ctx* ctx);
  * instead of being rebuilt on every call (the workspace must then be left untouched between the calls).
  * Setting the option (to either value) forgets what is cached. */
 #define QASR_OPT_STATIC_WEIGHTS 5
+/* Tuning aids (default 0 = the library chooses).  QASR_OPT_GEMM_FRAME_TILE: frames per work item of the
+ * pointwise tensor-core GEMM (a multiple of 16 in [16, 256]; at most 128 when C_in > 512).
+ * QASR_OPT_DW_FRAME_TILE: frames per window of the tensor-core depthwise kernel (a multiple of 16 in
+ * [16, 256]).  A value that does not fit the shape at hand is ignored for that call.  Results do not depend
+ * on either; they exist so that the built-in choice can be checked against the alternatives. */
+#define QASR_OPT_GEMM_FRAME_TILE 6
+#define QASR_OPT_DW_FRAME_TILE 7
 int qasr_set_option(qasr_ctx* ctx, int option, int value);
 
 /* One kernel launch seen in profile mode: which table layer it belongs to (-1 outside

@@ -486,6 +486,10 @@ int qasr_launch_dw_tc(qasr_ctx* ctx, const QasrDwArgs& a) {
         const double cost = (double)mt * (128.0 * nt * span / 8192.0 + 0.5 * kga + 400.0);
         if (cost < best) { best = cost; p.NT = nt; p.tiles = tiles; }
     }
+    if (ctx->force_dw_nt >= 16 && ctx->force_dw_nt <= 256 && ctx->force_dw_nt % 16 == 0 && ctx->force_dw_nt <= ((a.T_out + 15) & ~15)) {
+        p.NT = ctx->force_dw_nt;                  // tuning aid: the caller's frame tile instead of the cost model's
+        p.tiles = (a.T_out + p.NT - 1) / p.NT;
+    }
     if (!p.NT) return 0;
     p.MT = p.b_chunks > 1 ? p.tiles * p.b_chunks : (p.tiles + p.tpm - 1) / p.tpm;
     if ((long long)a.C * p.MT > 0x7fffffffLL) return 0;

@@ -420,9 +420,11 @@ int qasr_gemm_tc_init(qasr_ctx* ctx) {
 // free of shared-memory bank conflicts for 16-byte row accesses), as wide as the resident activation tile
 // allows, and the 128-channel output tiles of one frame tile are split over m_groups CTAs when there
 // are fewer frame tiles than SMs. Cost model: rounds of 128-channel tiles per SM x (BN + fixed cost).
-static void choose_tiles(int sm_count, int B, int T, int m_tiles, int nc_max, qasr::tc::GemmParams& p) {
+static void choose_tiles(int sm_count, int B, int T, int m_tiles, int nc_max, int forced_bn, qasr::tc::GemmParams& p) {
     double best = 1e30;
-    for (int bn = 48; bn <= 128 * nc_max; bn += 32) {           // 48, 80, 112, ... : odd multiples of 16
+    // forced_bn: the caller's frame tile (a tuning aid) instead of the search, if the kernel can take it
+    const bool forced = forced_bn >= 16 && forced_bn <= 128 * nc_max && forced_bn % 16 == 0;
+    for (int bn = forced ? forced_bn : 48; bn <= (forced ? forced_bn : 128 * nc_max); bn += 32) {   // 48, 80, 112, ... : odd multiples of 16
         const int tiles_t = (T + bn - 1) / bn;
         const long long n_tiles = (long long)B * tiles_t;
         for (int g = 1; g <= m_tiles; ++g) {
@@ -448,7 +450,7 @@ int qasr_launch_gemm_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
     memset(&p, 0, sizeof(p));
     p.B = a.B; p.C_in = a.C_in; p.C_out = a.C_out; p.T = a.T_out;
     p.m_tiles = (a.C_out + BM - 1) / BM;
-    choose_tiles(ctx->sm_count, a.B, a.T_out, p.m_tiles, a.C_in <= 512 ? 2 : 1, p);
+    choose_tiles(ctx->sm_count, a.B, a.T_out, p.m_tiles, a.C_in <= 512 ? 2 : 1, ctx->force_gemm_bn, p);
     p.n_items = a.B * p.tiles_t * p.m_groups;
     p.bias = a.bias; p.mult = a.mult; p.shift = a.shift; p.y = a.y; p.y32 = a.y_int32; p.relu = a.relu;
     p.terms = a.terms;

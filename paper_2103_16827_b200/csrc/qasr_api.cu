@@ -115,6 +115,12 @@ extern "C" int qasr_set_option(qasr_ctx* ctx, int option, int value) {
         case QASR_OPT_GRAPH: ctx->opt_graph = value != 0; break;
         case QASR_OPT_TENSOR_CORES: ctx->opt_tc = value != 0; break;
         case QASR_OPT_PROFILE: ctx->profiling = value != 0; break;
+        case QASR_OPT_GEMM_FRAME_TILE:
+        case QASR_OPT_DW_FRAME_TILE:
+            if (value != 0 && (value < 16 || value > 256 || value % 16 != 0))
+                QASR_FAIL(ctx, QASR_ERR_SHAPE, "frame tile %d must be 0 or a multiple of 16 in [16, 256]", value);
+            (option == QASR_OPT_GEMM_FRAME_TILE ? ctx->force_gemm_bn : ctx->force_dw_nt) = value;
+            break;
         case QASR_OPT_STATIC_WEIGHTS:
             ctx->opt_static_w = value != 0;
             ctx->prepared = false;

@@ -37,6 +37,7 @@ struct qasr_ctx {
     int sm_count = 148;
     int cc_major = 0;
     bool opt_graph = true, opt_tc = true, opt_pdl = true, opt_static_w = false;
+    int force_gemm_bn = 0, force_dw_nt = 0;      // tuning aids: 0 = automatic
     int64_t launches = 0;
     char err[512] = {0};
     // cached CUDA graph of the last qasr_encoder_forward call

@@ -724,6 +724,58 @@ def test_outputs_stay_inside_their_tensors_and_repeat_bit_for_bit(q, ctx, case):
     assert _guards_intact(raw, y.numel() * y.element_size()), "output guards"
 
 
+# ------------------------------------------------------------------ tile choices against their alternatives
+def _time_us(fn, ctx, iters=30):
+    for _ in range(3):
+        fn()
+    ctx.poll_status()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda._sleep(5_000_000)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters * 1e3
+
+
+@pytest.mark.parametrize("kind,dims", [("gemm", (32, 512, 512, 800)), ("gemm", (32, 256, 256, 800)), ("gemm", (32, 256, 512, 800)),
+                                       ("dw", (32, 512, 800, 75)), ("dw", (32, 256, 800, 33))])
+def test_built_in_frame_tile_is_close_to_the_best_alternative(q, ctx, kind, dims):
+    """The frame tiles come from small cost models with hand-set constants; at the benchmark's layer shapes the
+    built-in choice must be within 12 % of the fastest of the other tiles the kernel accepts (timed back to
+    back, device time), and every tile gives the same bits."""
+    rng = np.random.default_rng(17)
+    if kind == "gemm":
+        B, Ci, Co, T = dims
+        x = dev(rng.integers(-128, 128, size=(B, Ci, T)).astype(np.int8))
+        w = dev(rng.integers(-127, 128, size=(Co, Ci, 1)).astype(np.int8))
+        m, s = rand_rq(rng, Co, 24, 26)
+        md, sd = dev(m), dev(s)
+        y = torch.empty((B, Co, T), dtype=torch.int8, device="cuda")
+        fn = lambda: ctx.conv(x, w, None, 0, md, sd, True, y=y)
+        opt, tiles = q.OPT_GEMM_FRAME_TILE, [80, 112, 144, 176, 208, 240]
+    else:
+        B, C, T, K = dims
+        x = dev(rng.integers(-128, 128, size=(B, C, T)).astype(np.int8))
+        w = dev(rng.integers(-127, 128, size=(C, K)).astype(np.int8))
+        m, s = rand_rq(rng, C, 20, 22)
+        md, sd = dev(m), dev(s)
+        y = torch.empty((B, C, T), dtype=torch.int8, device="cuda")
+        fn = lambda: ctx.dw_conv(x, w, 1, 1, md, sd, y=y)
+        opt, tiles = q.OPT_DW_FRAME_TILE, [112, 144, 160, 208, 256]
+    t_auto = _time_us(fn, ctx)
+    want = y.clone()
+    best = None
+    for bn in tiles:
+        ctx.set_option(opt, bn)
+        t = _time_us(fn, ctx)
+        assert torch.equal(y, want), "tile %d changes the result" % bn
+        best = t if best is None else min(best, t)
+    ctx.set_option(opt, 0)
+    assert t_auto <= 1.12 * best, "built-in tile: %.2f us, best alternative: %.2f us" % (t_auto, best)
+
+
 # ------------------------------------------------------------------ errors are codes, not faults
 def test_argument_errors_return_codes(q, ctx):
     x = torch.zeros((1, 16, 64), dtype=torch.int8, device="cuda")
