@@ -328,6 +328,25 @@ int qasr_encoder_forward_host(qasr_ctx* ctx, const qasr_layer* table, int n_laye
                               void* workspace, size_t workspace_bytes,
                               int32_t* logits_q_host, float* logits_host, const float* out_scale);
 
+/* Pipelined host variant for callers that stream batch after batch (Sec. 3.2 deploys the encoder as a whole-model
+ * forward per call): qasr_encoder_forward_host_async only enqueues -- input copy, forward pass, result copies --
+ * and returns; the copies run on streams of the context's own, so that with two slots used in turn the copies of
+ * one call overlap the kernels of the other.  qasr_encoder_host_wait(slot) blocks until the results of the last
+ * call on that slot are in host memory (and returns at once if there is none).
+ *   - slot is 0 or 1; each has its own device staging, carved from the end of the workspace, so workspace_bytes
+ *     must be at least qasr_encoder_host_pipeline_bytes.  A call on a slot first waits (on the host) for that
+ *     slot's previous results.
+ *   - x_host, logits_q_host, logits_host: HOST pointers (pinned memory, else the copies are not asynchronous); they
+ *     must stay valid, and x_host unchanged, until qasr_encoder_host_wait(slot) has returned.
+ *   - The kernels run on the context's stream in call order; device errors surface through qasr_poll_status.
+ *   - Not usable while the context's stream is being captured. */
+int qasr_encoder_host_pipeline_bytes(const qasr_layer* table, int n_layers, int B, int C_in, int T, size_t* bytes);
+int qasr_encoder_forward_host_async(qasr_ctx* ctx, const qasr_layer* table, int n_layers,
+                                    const int8_t* x_host, int B, int C_in, int T,
+                                    void* workspace, size_t workspace_bytes,
+                                    int32_t* logits_q_host, float* logits_host, const float* out_scale, int slot);
+int qasr_encoder_host_wait(qasr_ctx* ctx, int slot);
+
 #ifdef __cplusplus
 }
 #endif

@@ -98,6 +98,12 @@ def lib():
     L.qasr_encoder_buffer_info.argtypes = [P(QasrLayer), ci, ci, ci, ci, ci, P(cs), P(ci), P(ci)]
     L.qasr_encoder_host_staging_bytes.argtypes = [P(QasrLayer), ci, ci, ci, ci, P(cs)]
     L.qasr_encoder_forward_host.argtypes = [vp, P(QasrLayer), ci, vp, ci, ci, ci, vp, cs, vp, vp, vp]
+    L.qasr_encoder_host_pipeline_bytes.argtypes = [P(QasrLayer), ci, ci, ci, ci, P(cs)]
+    L.qasr_encoder_host_pipeline_bytes.restype = ci
+    L.qasr_encoder_forward_host_async.argtypes = [vp, P(QasrLayer), ci, vp, ci, ci, ci, vp, cs, vp, vp, vp, ci]
+    L.qasr_encoder_forward_host_async.restype = ci
+    L.qasr_encoder_host_wait.argtypes = [vp, ci]
+    L.qasr_encoder_host_wait.restype = ci
     for name in ("qasr_create", "qasr_destroy", "qasr_poll_status", "qasr_set_option", "qasr_dw_conv", "qasr_conv",
                  "qasr_tcs_block_workspace_bytes", "qasr_tcs_block", "qasr_residual_requant_add",
                  "qasr_dequant_logits", "qasr_encoder_workspace_bytes", "qasr_encoder_forward",
@@ -326,6 +332,23 @@ class Context:
                                                         _ptr(logits_host),
                                                         _ptr(dm.out_scale) if logits_host is not None else None))
         return logits_q_host, logits_host
+
+
+    def encoder_host_pipeline_bytes(self, dm, B, T):
+        out = ctypes.c_size_t()
+        self._check(self._lib.qasr_encoder_host_pipeline_bytes(dm.table, dm.n_layers, B, dm.C_in, T, ctypes.byref(out)))
+        return out.value
+
+    def encoder_forward_host_async(self, dm, x_host, workspace, logits_q_host, logits_host=None, slot=0):
+        B, C_in, T = x_host.shape
+        self._check(self._lib.qasr_encoder_forward_host_async(self._h, dm.table, dm.n_layers, _ptr(x_host), B, C_in, T,
+                                                              _ptr(workspace), workspace.numel(), _ptr(logits_q_host),
+                                                              _ptr(logits_host),
+                                                              _ptr(dm.out_scale) if logits_host is not None else None,
+                                                              int(slot)))
+
+    def encoder_host_wait(self, slot):
+        self._check(self._lib.qasr_encoder_host_wait(self._h, int(slot)))
 
 
 class DeviceModel:

@@ -91,6 +91,15 @@ extern "C" int qasr_destroy(qasr_ctx* ctx) {
         cudaEventDestroy(r.e1);
     }
     if (ctx->capture_stream) cudaStreamDestroy(ctx->capture_stream);
+    if (ctx->copy_in) cudaStreamSynchronize(ctx->copy_in);
+    if (ctx->copy_out) cudaStreamSynchronize(ctx->copy_out);
+    for (int s = 0; s < 2; ++s) {
+        if (ctx->ev_in[s]) cudaEventDestroy(ctx->ev_in[s]);
+        if (ctx->ev_comp[s]) cudaEventDestroy(ctx->ev_comp[s]);
+        if (ctx->ev_out[s]) cudaEventDestroy(ctx->ev_out[s]);
+    }
+    if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
+    if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
     cudaFree(ctx->d_status);
     delete ctx;
     return QASR_OK;
@@ -763,7 +772,7 @@ extern "C" int qasr_encoder_forward(qasr_ctx* ctx, const qasr_layer* table, int 
     // Static-weights option: the regrouped weights in the workspace are those of this very call.
     QasrPlanKey key;
     qasr_plan_key(key, table, n_layers, x, B, C_in, T, workspace, logits_q, logits, out_scale);
-    const bool weights_ready = ctx->opt_static_w && ctx->prepared && ctx->prepared_key == key;
+    const bool weights_ready = ctx->opt_static_w && ctx->prepared && ctx->prepared_key.same_weights_home(key);
     if (ctx->opt_static_w && !weights_ready) {
         ctx->prepared_key = key;      // this call rebuilds them (stream order makes them ready for the next one)
         ctx->prepared = true;
@@ -772,12 +781,18 @@ extern "C" int qasr_encoder_forward(qasr_ctx* ctx, const qasr_layer* table, int 
         return enqueue_table(ctx, table, n_layers, p, x, B, (char*)workspace, logits_q, logits, out_scale, weights_ready);
 
     // Graph path: replay when the call is identical to the cached one, else capture it.
-    if (ctx->graph_exec && ctx->graph_key == key && ctx->graph_regroups == !weights_ready) {
-        QASR_CUDA(ctx, cudaGraphLaunch(ctx->graph_exec, ctx->stream));
-        ctx->launches += ctx->graph_nodes;
-        return QASR_OK;
+    for (qasr_ctx::GraphEntry& ge : ctx->graphs) {
+        if (ge.exec && ge.key == key && ge.regroups == !weights_ready) {
+            QASR_CUDA(ctx, cudaGraphLaunch(ge.exec, ctx->stream));
+            ctx->launches += ge.nodes;
+            ge.last_use = ++ctx->graph_tick;
+            return QASR_OK;
+        }
     }
-    qasr_plan_cache_clear(ctx);
+    // not cached: the least recently used entry makes room
+    qasr_ctx::GraphEntry& slot = ctx->graphs[ctx->graphs[0].last_use <= ctx->graphs[1].last_use ? 0 : 1];
+    if (slot.exec) cudaGraphExecDestroy(slot.exec);
+    slot = qasr_ctx::GraphEntry();
     cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
     QASR_CUDA(ctx, cudaStreamIsCapturing(ctx->stream, &cs));
     if (cs != cudaStreamCaptureStatusNone)  // the caller is capturing: just enqueue into their graph
@@ -801,14 +816,95 @@ extern "C" int qasr_encoder_forward(qasr_ctx* ctx, const qasr_layer* table, int 
         return rc;
     }
     QASR_CUDA(ctx, ce);
-    ce = cudaGraphInstantiate(&ctx->graph_exec, g, 0);
+    ce = cudaGraphInstantiate(&slot.exec, g, 0);
     cudaGraphDestroy(g);
+    if (ce != cudaSuccess) slot.exec = nullptr;
     QASR_CUDA(ctx, ce);
-    ctx->graph_key = key;
-    ctx->graph_nodes = nodes;
-    ctx->graph_regroups = !weights_ready;
-    QASR_CUDA(ctx, cudaGraphLaunch(ctx->graph_exec, ctx->stream));
+    slot.key = key;
+    slot.nodes = nodes;
+    slot.regroups = !weights_ready;
+    slot.last_use = ++ctx->graph_tick;
+    QASR_CUDA(ctx, cudaGraphLaunch(slot.exec, ctx->stream));
     ctx->launches += nodes;
+    return QASR_OK;
+}
+
+// Streams and events of the pipelined host entry point, created on first use.
+static int host_pipeline_init(qasr_ctx* ctx) {
+    if (ctx->copy_in) return QASR_OK;
+    QASR_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking));
+    QASR_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking));
+    for (int s = 0; s < 2; ++s) {
+        QASR_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_in[s], cudaEventDisableTiming));
+        QASR_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_comp[s], cudaEventDisableTiming));
+        QASR_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_out[s], cudaEventDisableTiming));
+    }
+    return QASR_OK;
+}
+
+extern "C" int qasr_encoder_host_pipeline_bytes(const qasr_layer* table, int n_layers, int B, int C_in, int T,
+                                                size_t* bytes) {
+    if (!bytes) return QASR_ERR_NULL;
+    TablePlan p;
+    int rc = plan_table(table, n_layers, B, C_in, T, p, nullptr, 0);
+    if (rc) return rc;
+    *bytes = p.total + 2 * staging_for(p, B, C_in, T).total;
+    return QASR_OK;
+}
+
+extern "C" int qasr_encoder_host_wait(qasr_ctx* ctx, int slot) {
+    if (!ctx) return QASR_ERR_NULL;
+    if (slot < 0 || slot > 1) QASR_FAIL(ctx, QASR_ERR_SHAPE, "slot %d must be 0 or 1", slot);
+    if (!ctx->slot_pending[slot]) return QASR_OK;
+    QASR_CUDA(ctx, cudaSetDevice(ctx->device));
+    QASR_CUDA(ctx, cudaEventSynchronize(ctx->ev_out[slot]));
+    ctx->slot_pending[slot] = false;
+    return QASR_OK;
+}
+
+extern "C" int qasr_encoder_forward_host_async(qasr_ctx* ctx, const qasr_layer* table, int n_layers,
+                                               const int8_t* x_host, int B, int C_in, int T,
+                                               void* workspace, size_t workspace_bytes,
+                                               int32_t* logits_q_host, float* logits_host, const float* out_scale,
+                                               int slot) {
+    if (!ctx) return QASR_ERR_NULL;
+    if (!x_host || !logits_q_host) QASR_FAIL(ctx, QASR_ERR_NULL, "qasr_encoder_forward_host_async: x or logits_q is NULL");
+    if (slot < 0 || slot > 1) QASR_FAIL(ctx, QASR_ERR_SHAPE, "slot %d must be 0 or 1", slot);
+    TablePlan p;
+    int rc = plan_table(table, n_layers, B, C_in, T, p, ctx->err, sizeof(ctx->err));
+    if (rc) return rc;
+    const Staging s = staging_for(p, B, C_in, T);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < p.total + 2 * s.total)
+        QASR_FAIL(ctx, QASR_ERR_WORKSPACE, "qasr_encoder_forward_host_async needs %zu bytes of 256-byte aligned workspace", p.total + 2 * s.total);
+    QASR_CUDA(ctx, cudaSetDevice(ctx->device));
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    QASR_CUDA(ctx, cudaStreamIsCapturing(ctx->stream, &cs));
+    if (cs != cudaStreamCaptureStatusNone) QASR_FAIL(ctx, QASR_ERR_CUDA, "qasr_encoder_forward_host_async cannot run inside a stream capture");
+    if ((rc = host_pipeline_init(ctx))) return rc;
+    // the slot's previous results must have reached the host before its device buffers are written again
+    if ((rc = qasr_encoder_host_wait(ctx, slot))) return rc;
+    char* st = (char*)workspace + p.total + (size_t)slot * s.total;
+    int8_t* x_dev = (int8_t*)(st + s.x);
+    int32_t* lq_dev = (int32_t*)(st + s.lq);
+    float* lf_dev = logits_host ? (float*)(st + s.lf) : nullptr;
+    const size_t n_logit = (size_t)B * p.C_last * p.T_last;
+    // input copy on its own stream: it may run while the kernels of the other slot's call still do
+    QASR_CUDA(ctx, cudaMemcpyAsync(x_dev, x_host, (size_t)B * C_in * T, cudaMemcpyHostToDevice, ctx->copy_in));
+    QASR_CUDA(ctx, cudaEventRecord(ctx->ev_in[slot], ctx->copy_in));
+    QASR_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev_in[slot], 0));
+    rc = qasr_encoder_forward(ctx, table, n_layers, x_dev, B, C_in, T, workspace, p.total, lq_dev, lf_dev,
+                              lf_dev ? out_scale : nullptr);
+    if (rc) return rc;
+    QASR_CUDA(ctx, cudaEventRecord(ctx->ev_comp[slot], ctx->stream));
+    // the next input copy into this slot must not overtake these kernels (the host-side wait above already
+    // orders it after them; this keeps the order on the device too)
+    QASR_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_in, ctx->ev_comp[slot], 0));
+    // result copies on a third stream: they overlap the next call's kernels
+    QASR_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_out, ctx->ev_comp[slot], 0));
+    QASR_CUDA(ctx, cudaMemcpyAsync(logits_q_host, lq_dev, n_logit * 4, cudaMemcpyDeviceToHost, ctx->copy_out));
+    if (lf_dev) QASR_CUDA(ctx, cudaMemcpyAsync(logits_host, lf_dev, n_logit * 4, cudaMemcpyDeviceToHost, ctx->copy_out));
+    QASR_CUDA(ctx, cudaEventRecord(ctx->ev_out[slot], ctx->copy_out));
+    ctx->slot_pending[slot] = true;
     return QASR_OK;
 }
 

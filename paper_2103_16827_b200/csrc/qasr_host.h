@@ -15,6 +15,11 @@ struct QasrPlanKey {
         return B == o.B && C_in == o.C_in && T == o.T && table == o.table &&
                std::memcmp(ptrs, o.ptrs, sizeof(ptrs)) == 0;
     }
+    // Same layer table, shape and workspace (whatever the input and output tensors are): the regrouped
+    // weights that one such call left in the workspace are the ones the other needs.
+    bool same_weights_home(const QasrPlanKey& o) const {
+        return B == o.B && C_in == o.C_in && T == o.T && ptrs[1] == o.ptrs[1] && table == o.table;
+    }
 };
 
 // kernel ids reported by the profiler
@@ -40,12 +45,22 @@ struct qasr_ctx {
     int force_gemm_bn = 0, force_dw_nt = 0;      // tuning aids: 0 = automatic
     int64_t launches = 0;
     char err[512] = {0};
-    // cached CUDA graph of the last qasr_encoder_forward call
-    cudaGraphExec_t graph_exec = nullptr;
+    // cached CUDA graphs of the last qasr_encoder_forward calls (two entries, least recently used one is
+    // replaced: a caller that alternates between two sets of buffers replays both)
+    struct GraphEntry {
+        cudaGraphExec_t exec = nullptr;
+        QasrPlanKey key;
+        int64_t nodes = 0;
+        bool regroups = true;        // the graph contains the weight regrouping kernels
+        uint64_t last_use = 0;
+    };
+    GraphEntry graphs[2];
+    uint64_t graph_tick = 0;
     cudaStream_t capture_stream = nullptr;
-    QasrPlanKey graph_key;
-    int64_t graph_nodes = 0;
-    bool graph_regroups = true;      // the cached graph contains the weight regrouping kernels
+    // pipelined host entry point: copy streams and per-slot events (created on first use)
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_comp[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
+    bool slot_pending[2] = {false, false};
     // static-weights option: the call whose regrouped weights the workspace currently holds
     QasrPlanKey prepared_key;
     bool prepared = false;
@@ -70,12 +85,10 @@ inline void qasr_plan_key(QasrPlanKey& k, const qasr_layer* table, int n, const 
 }
 
 inline void qasr_plan_cache_clear(qasr_ctx* ctx) {
-    if (ctx->graph_exec) {
-        cudaGraphExecDestroy(ctx->graph_exec);
-        ctx->graph_exec = nullptr;
+    for (qasr_ctx::GraphEntry& g : ctx->graphs) {
+        if (g.exec) cudaGraphExecDestroy(g.exec);
+        g = qasr_ctx::GraphEntry();
     }
-    ctx->graph_key = QasrPlanKey();
-    ctx->graph_nodes = 0;
 }
 
 // Brackets one kernel launch with events when the context is in profile mode, and counts it.

@@ -489,6 +489,40 @@ def test_encoder_forward_host_buffers(q, ctx):
     assert np.max(np.abs(lf.numpy() - wf)) <= 1e-6
 
 
+def test_encoder_forward_host_pipelined_over_two_slots(q, ctx):
+    """Five batches through the pipelined host entry point, slots used in turn, a different input each time:
+    every batch's logits are the oracle's, although the copies of one call overlap the kernels of the next and
+    both slots replay their own captured graph."""
+    model, x0 = _small_quartz(variant="live")
+    dm = q.DeviceModel(model, 0)
+    B, C, T = x0.shape
+    rng = workloads.rng_for(123)
+    xs = [x0] + [workloads.draw_input(rng, B, C, T) for _ in range(4)]
+    want = [oracle.encoder_forward(model, x, keep=False)[:2] for x in xs]
+    ws = torch.zeros(ctx.encoder_host_pipeline_bytes(dm, B, T), dtype=torch.uint8, device="cuda")
+    xh = [torch.from_numpy(x).pin_memory() for x in xs]
+    lq = [torch.zeros(want[0][0].shape, dtype=torch.int32).pin_memory() for _ in xs]
+    lf = [torch.zeros(want[0][1].shape, dtype=torch.float32).pin_memory() for _ in xs]
+    for i in range(len(xs)):
+        ctx.encoder_forward_host_async(dm, xh[i], ws, lq[i], lf[i], slot=i % 2)
+        if i >= 1:
+            ctx.encoder_host_wait((i - 1) % 2)
+            assert_same(lq[i - 1].numpy(), want[i - 1][0], "pipelined logits_q, batch %d" % (i - 1))
+    ctx.encoder_host_wait((len(xs) - 1) % 2)
+    ctx.encoder_host_wait(0)
+    ctx.encoder_host_wait(1)                    # nothing pending: returns at once
+    ctx.poll_status()
+    for i in range(len(xs)):
+        assert_same(lq[i].numpy(), want[i][0], "pipelined logits_q, batch %d" % i)
+        assert np.max(np.abs(lf[i].numpy() - want[i][1])) <= 1e-6
+    with pytest.raises(q.QasrError) as e:
+        ctx.encoder_forward_host_async(dm, xh[0], ws, lq[0], lf[0], slot=2)
+    assert e.value.code == -2
+    with pytest.raises(q.QasrError) as e:
+        ctx.encoder_forward_host_async(dm, xh[0], ws[:4096], lq[0], lf[0], slot=0)
+    assert e.value.code == -6
+
+
 def test_config2_full_batch_every_utterance(q, ctx):
     """QuartzNet-15x5 shape at B=32, T=1600 in the benchmark's launch configuration (ping-pong buffers, graph
     replay): the logits of all 32 utterances against the oracle."""
