@@ -4,6 +4,7 @@
   python -m paper_2103_16827_b200.microbench dw   B C T K [--stride S] [--dilation D]
   python -m paper_2103_16827_b200.microbench tcs  B C_in C_out T K
   python -m paper_2103_16827_b200.microbench add  B C T N_TERMS
+  python -m paper_2103_16827_b200.microbench peak [KBLOCKS]      (int8 tensor-core rate of this GPU)
 
 The launches are queued behind a short device-side delay so that they run back to back and the
 figure is device time per launch, not host launch latency.  Prints one JSON line.  This is also
@@ -26,8 +27,8 @@ def _dev(a):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("op", choices=["conv", "dw", "tcs", "add"])
-    ap.add_argument("dims", type=int, nargs="+")
+    ap.add_argument("op", choices=["conv", "dw", "tcs", "add", "peak"])
+    ap.add_argument("dims", type=int, nargs="*")
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--stride", type=int, default=1)
@@ -38,6 +39,12 @@ def main():
     args = ap.parse_args()
     rng = np.random.Generator(np.random.PCG64(0))
     ctx = Context(0)
+    if args.op == "peak":      # the int8 tensor-core rate of this GPU: dims = [K blocks per SM], default 2000 (~0.5 ms)
+        kb = args.dims[0] if args.dims else 2000
+        runs = [ctx.measure_int8_tensor_peak(kb) for _ in range(max(1, args.iters))]
+        print(json.dumps({"op": "peak", "kblocks": kb, "tops_best": max(r[0] for r in runs),
+                          "tops_median": sorted(r[0] for r in runs)[len(runs) // 2], "ms": runs[-1][1]}))
+        return
 
     def rq(C):
         return (_dev(rng.integers(1 << 14, 1 << 15, size=C).astype(np.int32)),

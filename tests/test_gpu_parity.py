@@ -758,6 +758,91 @@ def test_outputs_stay_inside_their_tensors_and_repeat_bit_for_bit(q, ctx, case):
     assert _guards_intact(raw, y.numel() * y.element_size()), "output guards"
 
 
+# ------------------------------------------------------------------ seeded random shapes
+def _random_cases(seed, n, kind):
+    rng = np.random.default_rng(seed)
+    cases = []
+    for _ in range(n):
+        big = rng.random() < 0.5                       # half of the cases qualify for the tensor-core kernels
+        B = int(rng.choice([8, 16, 24, 32])) if big else int(rng.integers(1, 6))
+        T = int(rng.integers(2, 40)) * 16 if big else int(rng.integers(1, 300))
+        stride = int(rng.choice([1, 1, 2]))
+        dil = int(rng.choice([1, 1, 2]))
+        if kind == "dw":
+            C = int(rng.integers(1, 48))
+            K = int(rng.choice([1, 3, 11, 33, 39, 51, 63, 75, 87]))
+            cases.append((B, C, T, K, stride, dil))
+        else:
+            Ci = int(rng.choice([64, 128, 192, 256])) if big else int(rng.integers(1, 80))
+            Co = int(rng.integers(1, 200))
+            K = int(rng.choice([1, 1, 1, 3, 5, 11]))
+            if K == 1 and rng.random() < 0.7:
+                stride = dil = 1
+            cases.append((B, Ci, Co, T, K, stride, dil))
+    return cases
+
+
+def test_dw_conv_random_shapes(q, ctx):
+    """Forty seeded random depthwise problems (batch, channels, length, taps, stride, dilation), half of them in
+    the tensor-core kernel's domain, half ragged: every one bit-exact against the oracle."""
+    rng = np.random.default_rng(2024)
+    seen = set()
+    for B, C, T, K, stride, dil in _random_cases(31, 40, "dw"):
+        x = rng.integers(-128, 128, size=(B, C, T)).astype(np.int8)
+        w = rng.integers(-127, 128, size=(C, K)).astype(np.int8)
+        m, s = rand_rq(rng, C, 17, 24)
+        want = oracle.requant(oracle.conv1d(x, w, None, stride, dil, depthwise=True), m, s)
+        got, kernels = _profiled(q, ctx, lambda: ctx.dw_conv(dev(x), dev(w), stride, dil, dev(m), dev(s)))
+        assert_same(got, want, "dw random %s" % ((B, C, T, K, stride, dil),))
+        seen.update(kernels)
+    assert "dw_conv_tc" in seen and len(seen) >= 2, seen
+
+
+def test_conv_random_shapes(q, ctx):
+    """Forty seeded random pointwise / K-tap convolutions with bias, ReLU or residual terms, scratch lent so that
+    the implicit-GEMM kernel takes what it can: every one bit-exact against the oracle, and all three convolution
+    kernels get used."""
+    rng = np.random.default_rng(2025)
+    seen = set()
+    for B, Ci, Co, T, K, stride, dil in _random_cases(32, 40, "conv"):
+        x = rng.integers(-128, 128, size=(B, Ci, T)).astype(np.int8)
+        w = rng.integers(-127, 128, size=(Co, Ci, K)).astype(np.int8)
+        bias = rng.integers(-4096, 4097, size=Co).astype(np.int32)
+        sh = max(2, int(np.ceil(np.log2(np.sqrt(Ci * K) * 73 * 74 * 2 ** 14.5 / 40))))
+        m, s = rand_rq(rng, Co, sh - 1, sh + 1)
+        acc = oracle.conv1d(x, w, bias, stride, dil)
+        ctx.set_conv_scratch(torch.zeros(max(256, ctx.conv_scratch_bytes(B, Ci, Co, T, K, stride)), dtype=torch.uint8, device="cuda"))
+        n_res = int(rng.integers(0, 3))
+        if n_res:
+            res = [rng.integers(-128, 128, size=acc.shape).astype(np.int8) for _ in range(n_res)]
+            tm = rng.integers(1 << 13, 1 << 15, size=n_res + 1).astype(np.int32)
+            ts = rng.integers(13, 17, size=n_res + 1).astype(np.uint8)
+            want = oracle.residual_add([oracle.requant(acc, m, s)] + res, tm, ts, relu=True)
+            run = lambda: ctx.conv(dev(x), dev(w), dev(bias), 4096, dev(m), dev(s), True, stride, dil,
+                                   terms=[None] + [dev(r) for r in res], term_mult=tm, term_shift=ts)
+        else:
+            relu = bool(rng.integers(0, 2))
+            want = oracle.requant(acc, m, s, relu=relu)
+            run = lambda: ctx.conv(dev(x), dev(w), dev(bias), 4096, dev(m), dev(s), relu, stride, dil)
+        got, kernels = _profiled(q, ctx, run)
+        ctx.set_conv_scratch(None)
+        assert_same(got, want, "conv random %s" % ((B, Ci, Co, T, K, stride, dil),))
+        seen.update(k for k in kernels if k != "conv_tc_prepare")
+    assert {"gemm_i8_tc", "conv_i8_tc", "conv_generic"} <= seen, seen
+
+
+def test_int8_tensor_peak_loop_reports_a_plausible_rate(q, ctx):
+    """The library's tcgen05 saturation loop: finishes, reports a rate between a tenth of and somewhat above the
+    nominal dense int8 figure, leaves a clean status, and refuses sizes outside its documented range."""
+    tops, ms = ctx.measure_int8_tensor_peak(2000)
+    assert ms > 0 and 450.0 < tops < 6000.0, (tops, ms)
+    ctx.poll_status()
+    for bad in (0, (1 << 20) + 1):
+        with pytest.raises(q.QasrError) as e:
+            ctx.measure_int8_tensor_peak(bad)
+        assert e.value.code == -2
+
+
 # ------------------------------------------------------------------ tile choices against their alternatives
 def _time_us(fn, ctx, iters=30):
     for _ in range(3):
