@@ -105,6 +105,11 @@ int qasr_poll_status(qasr_ctx* ctx);
  * on either; they exist so that the built-in choice can be checked against the alternatives. */
 #define QASR_OPT_GEMM_FRAME_TILE 6
 #define QASR_OPT_DW_FRAME_TILE 7
+/* QASR_OPT_SIDE_BRANCH (default 1): inside the captured graph of qasr_encoder_forward a pointwise layer whose
+ * output the next layer does not read (a block's residual projection) runs beside the main chain, on the SMs the
+ * main chain's kernels leave idle, and is joined in front of the first layer that needs it.  Results do not depend
+ * on the option. */
+#define QASR_OPT_SIDE_BRANCH 8
 int qasr_set_option(qasr_ctx* ctx, int option, int value);
 
 /* One kernel launch seen in profile mode: which table layer it belongs to (-1 outside

@@ -486,7 +486,7 @@ int qasr_launch_conv_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
         for (int g = 1; g <= p.m_tiles; ++g) {
             const int per = (p.m_tiles + g - 1) / g;
             if ((p.m_tiles + per - 1) / per != g) continue;
-            const long long rounds = (n_tiles * g + ctx->sm_count - 1) / ctx->sm_count;
+            const long long rounds = (n_tiles * g + qasr_grid_slots(ctx) - 1) / qasr_grid_slots(ctx);
             const double blk = (bn > 176 ? bn : 176) + (double)R * P / a.K;
             const double cost = (double)rounds * per * blk + g * 1e-3;
             if (cost < best) {
@@ -567,7 +567,7 @@ int qasr_launch_conv_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
         }
     }
     const size_t smem = fixed + (size_t)p.x_stages * p.x_stage_bytes + (size_t)p.w_stages * CV_W_STAGE_BYTES;
-    const int grid = p.n_items < ctx->sm_count ? p.n_items : ctx->sm_count;
+    const int grid = p.n_items < qasr_grid_slots(ctx) ? p.n_items : qasr_grid_slots(ctx);
     QasrLaunchScope ls(ctx, QASR_K_CONV_TC, qasr_conv_macs(a), qasr_conv_bytes(a));
     cudaError_t e = qasr_launch_overlapped(ctx, conv_i8_tc_kernel, dim3(grid), dim3(CV_THREADS), smem, tmW, tmX, tmY, p);
     if (e != cudaSuccess) {

@@ -548,7 +548,7 @@ int qasr_launch_dw_tc(qasr_ctx* ctx, const QasrDwArgs& a) {
         box[0] = (cuuint32_t)(narrow > 0 ? narrow : p.stage_w);
         if (!qasr_encode_map_u8(ctx, &tmY, a.y, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE)) return QASR_ERR_CUDA;
     }
-    const int grid = p.n_items < ctx->sm_count ? p.n_items : ctx->sm_count;
+    const int grid = p.n_items < qasr_grid_slots(ctx) ? p.n_items : qasr_grid_slots(ctx);
     QasrLaunchScope ls(ctx, QASR_K_DW_TC, qasr_dw_macs(a), qasr_dw_bytes(a));
     cudaError_t e = qasr_launch_overlapped(ctx, dw_tc_kernel, dim3(grid), dim3(THREADS), smem, tmX, tmY, tmYw, p);
     if (e != cudaSuccess) {

@@ -450,7 +450,7 @@ int qasr_launch_gemm_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
     memset(&p, 0, sizeof(p));
     p.B = a.B; p.C_in = a.C_in; p.C_out = a.C_out; p.T = a.T_out;
     p.m_tiles = (a.C_out + BM - 1) / BM;
-    choose_tiles(ctx->sm_count, a.B, a.T_out, p.m_tiles, a.C_in <= 512 ? 2 : 1, ctx->force_gemm_bn, p);
+    choose_tiles(qasr_grid_slots(ctx), a.B, a.T_out, p.m_tiles, a.C_in <= 512 ? 2 : 1, ctx->force_gemm_bn, p);
     p.n_items = a.B * p.tiles_t * p.m_groups;
     p.bias = a.bias; p.mult = a.mult; p.shift = a.shift; p.y = a.y; p.y32 = a.y_int32; p.relu = a.relu;
     p.terms = a.terms;
@@ -498,7 +498,7 @@ int qasr_launch_gemm_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
         tmYw = tmX;
     }
     const size_t smem = fixed + (size_t)p.w_stages * BM * BK;
-    const int grid = p.n_items < ctx->sm_count ? p.n_items : ctx->sm_count;
+    const int grid = p.n_items < qasr_grid_slots(ctx) ? p.n_items : qasr_grid_slots(ctx);
     QasrLaunchScope ls(ctx, QASR_K_GEMM_TC, qasr_conv_macs(a), qasr_conv_bytes(a));
     cudaError_t e = BK == 128
         ? qasr_launch_overlapped(ctx, gemm_i8_tc_kernel<128>, dim3(grid), dim3(THREADS), smem, tmW, tmX, tmXl, tmY, tmYw, p)

@@ -91,6 +91,9 @@ extern "C" int qasr_destroy(qasr_ctx* ctx) {
         cudaEventDestroy(r.e1);
     }
     if (ctx->capture_stream) cudaStreamDestroy(ctx->capture_stream);
+    if (ctx->side_stream) cudaStreamDestroy(ctx->side_stream);
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    if (ctx->ev_side) cudaEventDestroy(ctx->ev_side);
     if (ctx->copy_in) cudaStreamSynchronize(ctx->copy_in);
     if (ctx->copy_out) cudaStreamSynchronize(ctx->copy_out);
     for (int s = 0; s < 2; ++s) {
@@ -124,6 +127,7 @@ extern "C" int qasr_set_option(qasr_ctx* ctx, int option, int value) {
         case QASR_OPT_GRAPH: ctx->opt_graph = value != 0; break;
         case QASR_OPT_TENSOR_CORES: ctx->opt_tc = value != 0; break;
         case QASR_OPT_PROFILE: ctx->profiling = value != 0; break;
+        case QASR_OPT_SIDE_BRANCH: ctx->opt_side = value != 0; break;
         case QASR_OPT_GEMM_FRAME_TILE:
         case QASR_OPT_DW_FRAME_TILE:
             if (value != 0 && (value < 16 || value > 256 || value % 16 != 0))
@@ -660,16 +664,60 @@ extern "C" int qasr_encoder_host_staging_bytes(const qasr_layer* table, int n_la
 // Enqueue every layer of a validated table (no graph handling here).
 static int enqueue_table(qasr_ctx* ctx, const qasr_layer* tb, int n, const TablePlan& p,
                          const int8_t* x, int B, char* ws, int32_t* logits_q, float* logits,
-                         const float* out_scale, bool weights_ready = false) {
+                         const float* out_scale, bool weights_ready = false, bool capturing = false) {
     auto buf_ptr = [&](int id) -> int8_t* { return id == 0 ? const_cast<int8_t*>(x) : (int8_t*)(ws + p.bufs[id].offset); };
     // Shapes of buffers change as layers overwrite them, so they are re-tracked here.
     std::vector<int> curC(p.bufs.size(), 0);
     curC[0] = p.bufs[0].C;
+    // Side branch (only while the table is being captured into a graph): a pointwise convolution whose result
+    // the next layer does not read -- a block's residual projection; several in a row for dense residuals -- runs
+    // on a second stream with a small grid, on the SMs that the main chain's 128-item kernels leave idle, and joins
+    // the main chain in front of the first layer that reads one of its outputs or overwrites one of its tensors.
+    // While a branch is pending the main chain's persistent kernels launch 128 CTAs (their item counts are
+    // multiples of 128 at these shapes anyway). The branch's kernels follow one another in stream order.
+    struct {
+        bool pending = false;
+        std::vector<int> in_bufs, out_bufs;      // tensors the pending branch reads / writes
+        bool reads(int b) const { for (int v : in_bufs) if (v == b) return true; return false; }
+        bool writes(int b) const { for (int v : out_bufs) if (v == b) return true; return false; }
+    } side;
+    const int main_slots = 128;
+    const bool side_ok = capturing && ctx->opt_side && ctx->opt_tc && ctx->encode_tiled && !ctx->profiling &&
+                         ctx->sm_count >= main_slots + 16;
+    auto join_side = [&]() -> int {
+        if (!side.pending) return QASR_OK;
+        QASR_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev_side, 0));
+        side.pending = false;
+        side.in_bufs.clear();
+        side.out_bufs.clear();
+        ctx->grid_cap = 0;
+        return QASR_OK;
+    };
     for (int li = 0; li < n; ++li) {
         const qasr_layer& L = tb[li];
         const int T_i = p.t_in[li], T_o = p.t_out[li];
         int rc = QASR_OK;
         ctx->cur_layer = li;
+        // Does this layer go to the side branch? A pointwise layer on the tensor-core GEMM path whose output the
+        // next layer neither reads nor overwrites, while the main chain's kernels fit 128 CTAs.
+        bool to_side = false;
+        if (side_ok && L.kind == QASR_LAYER_PW && !L.out_int32 && L.n_terms == 0 && li + 2 < n &&
+            qasr_conv_shape_fits_gemm(L.C_in, 1, 1, 1, T_o) && (long long)B * ((T_o + 207) / 208) <= main_slots) {
+            const qasr_layer& N = tb[li + 1];
+            bool next_reads = N.kind != QASR_LAYER_ADD && N.in_buf == L.out_buf;
+            for (int j = (N.kind == QASR_LAYER_ADD ? 0 : 1); j < N.n_terms; ++j)
+                if (N.term_buf[j] == L.out_buf) next_reads = true;
+            to_side = !next_reads && N.out_buf != L.out_buf && N.out_buf != L.in_buf;
+        }
+        if (side.pending && !to_side) {
+            // join in front of a main-chain layer that reads one of the branch's outputs or writes one of its
+            // tensors (a layer that itself joins the branch follows the pending kernels in stream order)
+            bool hazard = side.reads(L.out_buf) || side.writes(L.out_buf) || L.out_int32;
+            if (L.kind != QASR_LAYER_ADD && side.writes(L.in_buf)) hazard = true;
+            for (int j = (L.kind == QASR_LAYER_ADD ? 0 : 1); j < L.n_terms; ++j)
+                if (side.writes(L.term_buf[j])) hazard = true;
+            if (hazard && (rc = join_side())) return rc;
+        }
         if (L.kind == QASR_LAYER_ADD) {
             QasrTerms t;
             memset(&t, 0, sizeof(t));
@@ -723,7 +771,25 @@ static int enqueue_table(qasr_ctx* ctx, const qasr_layer* tb, int n, const Table
                 a.terms.mult[j] = L.term_mult[j];
                 a.terms.shift[j] = L.term_shift[j];
             }
-            if (L.kind == QASR_LAYER_TCS) {
+            if (to_side) {
+                if (!ctx->side_stream) QASR_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->side_stream, cudaStreamNonBlocking));
+                if (!ctx->ev_fork) QASR_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming));
+                if (!ctx->ev_side) QASR_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_side, cudaEventDisableTiming));
+                a.T = T_i; a.T_out = T_o; a.K = 1; a.stride = 1; a.dilation = 1;
+                QASR_CUDA(ctx, cudaEventRecord(ctx->ev_fork, ctx->stream));
+                QASR_CUDA(ctx, cudaStreamWaitEvent(ctx->side_stream, ctx->ev_fork, 0));
+                cudaStream_t main_stream = ctx->stream;
+                ctx->stream = ctx->side_stream;
+                ctx->grid_cap = ctx->sm_count - main_slots;
+                rc = run_conv(ctx, a);
+                ctx->stream = main_stream;
+                ctx->grid_cap = main_slots;
+                if (rc) return rc;
+                QASR_CUDA(ctx, cudaEventRecord(ctx->ev_side, ctx->side_stream));
+                side.pending = true;
+                side.in_bufs.push_back(L.in_buf);
+                side.out_bufs.push_back(L.out_buf);
+            } else if (L.kind == QASR_LAYER_TCS) {
                 QasrDwArgs d{in, L.w_dw, L.rq_dw.mult, L.rq_dw.shift, nullptr, B, L.C_in, T_i, T_o, L.K, L.stride, L.dilation};
                 a.T = T_o; a.T_out = T_o; a.K = 1; a.stride = 1; a.dilation = 1;
                 rc = run_tcs(ctx, d, a, ws + p.scratch_offset);
@@ -742,6 +808,10 @@ static int enqueue_table(qasr_ctx* ctx, const qasr_layer* tb, int n, const Table
     }
     ctx->cur_layer = -1;
     memset(&ctx->prefetch, 0, sizeof(ctx->prefetch));
+    {
+        int rcj = join_side();
+        if (rcj) return rcj;
+    }
     if (logits && out_scale) {
         QasrLaunchScope ls(ctx, QASR_K_DEQUANT, 0, (double)B * p.C_last * p.T_last * 8);
         QASR_CUDA(ctx, qasr_launch_dequant(logits_q, B, p.C_last, p.T_last, out_scale, logits, ctx->stream));
@@ -805,8 +875,9 @@ extern "C" int qasr_encoder_forward(qasr_ctx* ctx, const qasr_layer* table, int 
     const int64_t before = ctx->launches;
     cudaStream_t user_stream = ctx->stream;
     ctx->stream = ctx->capture_stream;
-    rc = enqueue_table(ctx, table, n_layers, p, x, B, (char*)workspace, logits_q, logits, out_scale, weights_ready);
+    rc = enqueue_table(ctx, table, n_layers, p, x, B, (char*)workspace, logits_q, logits, out_scale, weights_ready, true);
     ctx->stream = user_stream;
+    ctx->grid_cap = 0;
     cudaGraph_t g = nullptr;
     cudaError_t ce = cudaStreamEndCapture(ctx->capture_stream, &g);
     const int64_t nodes = ctx->launches - before;

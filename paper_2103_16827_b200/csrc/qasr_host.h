@@ -43,6 +43,12 @@ struct qasr_ctx {
     int cc_major = 0;
     bool opt_graph = true, opt_tc = true, opt_pdl = true, opt_static_w = false;
     int force_gemm_bn = 0, force_dw_nt = 0;      // tuning aids: 0 = automatic
+    // Side branch of a captured layer table: a convolution whose result is needed only several layers later
+    // (a block's residual projection) runs on a second stream, on the SMs the main chain leaves idle.
+    bool opt_side = true;
+    int grid_cap = 0;                            // > 0: persistent kernels launch at most this many CTAs
+    cudaStream_t side_stream = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_side = nullptr;
     int64_t launches = 0;
     char err[512] = {0};
     // cached CUDA graphs of the last qasr_encoder_forward calls (two entries, least recently used one is
@@ -128,6 +134,11 @@ inline bool qasr_terms_fit_int32(const QasrTerms& t) {
         sum += ((128LL * t.mult[j]) >> t.shift[j]) + 1;
     }
     return sum < (1LL << 31);
+}
+
+// CTAs a one-CTA-per-SM persistent kernel may launch: every SM, unless a side branch shares the GPU.
+inline int qasr_grid_slots(const qasr_ctx* ctx) {
+    return ctx->grid_cap > 0 && ctx->grid_cap < ctx->sm_count ? ctx->grid_cap : ctx->sm_count;
 }
 
 // Launches a kernel whose prologue may overlap the tail of the previous kernel in the stream

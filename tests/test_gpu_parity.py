@@ -474,6 +474,49 @@ def test_config1_pingpong_buffers_and_graph_replay(q, ctx):
     assert_same(lq, wq, "logits_q generic kernels")
 
 
+@pytest.mark.parametrize("which", ["quartznet", "quartznet_recycled_block_input", "jasper"])
+def test_side_branch_of_residual_projections_changes_no_bit(q, ctx, which):
+    """Inside the captured graph the residual projections run beside the main chain (QASR_OPT_SIDE_BRANCH, on by
+    default). With the option on and off the logits are the oracle's, for QuartzNet blocks (one projection per
+    block), for a table that recycles the block input's buffer while the projection may still read it (the
+    library must then join early) and for Jasper's dense residuals (several projections in a row on the branch)."""
+    if which == "jasper":
+        model, x = workloads.jasper_model(8, 416, variant="live", seed=7, mel=16, channels=(64, 64, 128), kernels=(11, 13, 17),
+                                          c1=64, k1=11, c2=128, k2=29, c3=128, n_out=29, subblocks=2)
+    else:
+        model, x = workloads.quartznet_model(8, 832, repeat=2, variant="live", seed=9, mel=16, channels=(64, 128), kernels=(33, 39),
+                                             c1=64, c2=128, c3=128, n_out=29, subblocks=3)
+    if which == "quartznet_recycled_block_input":
+        # from the second sub-block of every block on, the block input's buffer and that sub-block's output buffer
+        # exchange their names: the second sub-block then overwrites the tensor the projection reads
+        layers = model["layers"]
+        ren = lambda v, a, b: b if v == a else a if v == b else v
+        for i, L in enumerate(layers):
+            if L["name"].endswith(".res"):
+                a, b = L["in"], layers[i + 2]["out"]
+                for M in layers[i + 2:]:
+                    for key in ("in", "out"):
+                        if key in M:
+                            M[key] = ren(M[key], a, b)
+                    if M.get("res"):
+                        M["res"] = [ren(r, a, b) for r in M["res"]]
+    wq, wf, _ = oracle.encoder_forward(model, x, keep=False)
+    dm = q.DeviceModel(model, 0)
+    B, _, T = x.shape
+    ws = torch.zeros(max(ctx.encoder_workspace_bytes(dm, B, T), 256), dtype=torch.uint8, device="cuda")
+    lq = torch.zeros(wq.shape, dtype=torch.int32, device="cuda")
+    lf = torch.zeros(wf.shape, dtype=torch.float32, device="cuda")
+    xd = dev(x)
+    for side in (1, 0, 1):
+        ctx.set_option(q.OPT_SIDE_BRANCH, side)
+        for _ in range(2):                     # capture, then replay
+            lq.zero_()
+            ctx.encoder_forward(dm, xd, ws, lq, lf)
+            ctx.poll_status()
+            assert_same(lq, wq, "logits_q, %s, side branch %d" % (which, side))
+    assert np.max(np.abs(lf.cpu().numpy() - wf)) <= 1e-6
+
+
 def test_encoder_forward_host_buffers(q, ctx):
     model, x = _small_quartz(variant="live")
     wq, wf, _ = oracle.encoder_forward(model, x, keep=False)

@@ -222,8 +222,12 @@ def quartznet_model(B, T, repeat=1, variant="live", seed=1, mel=64, unique_bufs=
                 last = s == subblocks - 1
                 nxt = bld.tcs("%s.%d" % (tag, s), h, cin if s == 0 else c, c, k, 1, 1, True, MS_RELU,
                               res=[rbuf] if last else None)
-                bld.release(h)
+                if h != cur:
+                    bld.release(h)
                 h = nxt
+            # the block input keeps its buffer until the block ends: the projection that reads it may then run
+            # beside the sub-blocks instead of in front of them (nothing overwrites its input meanwhile)
+            bld.release(cur)
             bld.release(rbuf)
             cur = h
             cin = c
