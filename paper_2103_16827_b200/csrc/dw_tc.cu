@@ -195,7 +195,10 @@ dw_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
     if (warp == MMA_WARP) prefetch_ranges_l2(p.next, lane);
     // everything above touched only this CTA's own state and constants; from here on the previous kernel's output is read
     ptx::grid_dep_launch();
-    ptx::grid_dep_wait();
+    // The builders put the dependency wait off: taps, tap line and band of their first item depend only on the
+    // layer's constants and are built while the previous kernel drains (that item's window loads are issued by
+    // the epilogue warps, which do wait here); a builder waits before the first window load of its own.
+    if (warp >= BUILD_WARPS) ptx::grid_dep_wait();
 
     if (warp < BUILD_WARPS) {
         // ------------------------------------------------------------------ builders
@@ -219,7 +222,9 @@ dw_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
                                      (tile0 + at.ti) * p.NT * p.stride - p.padL + 128 * at.kb, c, b0, ptx::smem_u32(&sh->full[grp]));
             };
             const bool first_use = n == (uint32_t)grp;     // the stage has never been used: nothing to wait for
-            if (first_use) load_windows();                  // the bytes may land before tid 0 announces them
+            // the first item's boxes are issued by the epilogue warps, which have nothing to do yet (one box per
+            // warp side by side instead of three per builder warp one after the other); the bytes may land
+            // before tid 0 announces them
             if (tid < p.K) taps[tid] = tap_next;
             tap_next = fetch_tap(n + 2);
             asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "n"(BUILD_GROUP_THREADS) : "memory");   // taps staged
@@ -244,7 +249,10 @@ dw_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
             }
             asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "n"(BUILD_GROUP_THREADS) : "memory");   // tap line complete, go/no-go known
             if (!sh->build_ok[grp]) break;
-            if (!first_use) load_windows();
+            if (!first_use) {
+                ptx::grid_dep_wait();       // returns at once after the first time
+                load_windows();
+            }
             // Bt band: row nn holds the taps starting at byte nn*stride + lead. K-major with the 128-byte
             // swizzle: 16-byte chunk kc of row nn lives in K block kc / 8 at row nn, chunk (kc % 8) ^ (nn % 8).
             {
@@ -352,6 +360,27 @@ dw_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
         const int sti = srow / p.rows_b;
         const int srb = srow - sti * p.rows_b;
         const bool storer = p.staged && my_w > 0 && lane * p.box_rows < 32;
+        {
+            // window loads of the two builder groups' first items: box j of group g by epilogue thread
+            // (warp j % EPI_WARPS, lane j / EPI_WARPS) counting over both groups
+            const int ew = warp - BUILD_WARPS;
+            for (int g = 0; g < 2; ++g) {
+                const long long it64 = (long long)blockIdx.x + (long long)g * gridDim.x;
+                if (it64 >= p.n_items) break;
+                const int item = (int)it64;
+                const int c0 = item / p.MT;
+                int tile0, b0;
+                mtile_coords(p, item - c0 * p.MT, tile0, b0);
+                const int n_tiles = min(p.tpm, p.tiles - tile0);
+                const int n_boxes = n_tiles * p.a_kblocks;
+                uint8_t* const Astage = g ? A1 : A0;
+                for (int j = lane * EPI_WARPS + ew - g * 0; j < n_boxes; j += 32 * EPI_WARPS) {
+                    const int kb = j / n_tiles, ti = j - kb * n_tiles;
+                    ptx::tma_load_3d(ptx::smem_u32(Astage + kb * A_KBLOCK_BYTES + ti * p.rows_b * 128), &tmX,
+                                     (tile0 + ti) * p.NT * p.stride - p.padL + 128 * kb, c0, b0, ptx::smem_u32(&sh->full[g]));
+                }
+            }
+        }
         uint32_t n = (uint32_t)egrp;
         bool ok = true;
         // the requantisation constants of this group's next item are fetched while this one is requantised
