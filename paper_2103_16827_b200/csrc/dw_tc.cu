@@ -22,7 +22,10 @@
 // Bt) while the MMA warp issues the current stage and 8 epilogue warps requantise the previous
 // accumulator (per-channel scalar constants) and store 16 output frames per thread and step.  The taps
 // of a group's next item are fetched one item ahead (the first ones before the dependency wait): they
-// are constants of the layer whose first touch comes from DRAM.
+// are constants of the layer whose first touch comes from DRAM.  The first item of each builder group is
+// started differently: its band depends on constants only and is built without waiting for the previous
+// kernel, and its window loads are issued by the epilogue warps (idle at that point), one box per warp
+// side by side, as soon as their dependency wait returns.
 #include <cstdio>
 #include <cstring>
 
@@ -374,7 +377,7 @@ dw_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
                 const int n_tiles = min(p.tpm, p.tiles - tile0);
                 const int n_boxes = n_tiles * p.a_kblocks;
                 uint8_t* const Astage = g ? A1 : A0;
-                for (int j = lane * EPI_WARPS + ew - g * 0; j < n_boxes; j += 32 * EPI_WARPS) {
+                for (int j = lane * EPI_WARPS + ew; j < n_boxes; j += 32 * EPI_WARPS) {
                     const int kb = j / n_tiles, ti = j - kb * n_tiles;
                     ptx::tma_load_3d(ptx::smem_u32(Astage + kb * A_KBLOCK_BYTES + ti * p.rows_b * 128), &tmX,
                                      (tile0 + ti) * p.NT * p.stride - p.padL + 128 * kb, c0, b0, ptx::smem_u32(&sh->full[g]));
