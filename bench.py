@@ -42,6 +42,9 @@ def parse_args():
     ap.add_argument("--sustained-seconds", type=float, default=2.0,
                     help="length of the back-to-back replay run reported as `sustained` (0 = skip)")
     ap.add_argument("--no-int8-peak", action="store_true", help="skip the tcgen05 int8 saturation loop")
+    ap.add_argument("--no-side-branch", action="store_true",
+                    help="launch the residual projections in table order on the main chain (QASR_OPT_SIDE_BRANCH = 0); "
+                         "for launch lists whose per-kernel times are to be compared with the kernel-by-kernel pass")
     ap.add_argument("--static-weights", dest="static_weights", action="store_true", default=True,
                     help="promise the library that neither the weights nor the workspace change between steps: K-tap layers "
                          "then keep their regrouped weights (default; an inference benchmark's weights are constants)")
@@ -258,6 +261,8 @@ def run_ours(args):
     ctx = q.Context(local)
     if args.static_weights:
         ctx.set_option(q.OPT_STATIC_WEIGHTS, 1)
+    if args.no_side_branch:
+        ctx.set_option(q.OPT_SIDE_BRANCH, 0)
     last = model["layers"][-1]
     T_last = workloads.model_stats(model)["T_out"]      # frames of the last layer (strides differ per model)
     need = ctx.encoder_workspace_bytes(dm, B, T) + ctx.encoder_host_staging_bytes(dm, B, T)
@@ -403,7 +408,7 @@ def run_ours(args):
         for _ in range(3):
             step()
         off_ms, _ = timed(step, min(args.steps, 30))
-        ctx.set_option(q.OPT_SIDE_BRANCH, 1)
+        ctx.set_option(q.OPT_SIDE_BRANCH, 0 if args.no_side_branch else 1)
         for _ in range(3):
             step()
         ablation = {"side_branch_off_ms_per_step": off_ms / min(args.steps, 30),
@@ -527,7 +532,7 @@ def run_ours(args):
             "config": {"workload": "config %d: %s B=%d T=%d mel=%d (%s scales)" % (args.config, model["name"], B, T, C_in, args.variant),
                        "per_gpu_batch": B, "layers": len(model["layers"]),
                        "l2": "256 MiB buffer written between timed steps (outside the events)",
-                       "static_weights": bool(args.static_weights),
+                       "static_weights": bool(args.static_weights), "side_branch": not args.no_side_branch,
                        "parallelism": "replicas x%d, no collective" % world},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
             "roofline_depthwise": roofline_depthwise, "roofline_by_kind": roofline_by_kind,
