@@ -203,9 +203,9 @@ TRAFFIC = {
     "gemm_i8_tc": {"bytes_per_launch": 13.52e6, "source": "paper_2103_16827_b200/csrc/gemm_tc.cu",
                    "sha1": "997be66518dcc5bc52cbc10c5f332fb04e494dc2", "config": 2},
     "dw_conv_tc": {"bytes_per_launch": 13.20e6, "source": "paper_2103_16827_b200/csrc/dw_tc.cu",
-                   "sha1": "ca47bb3d387106f1e8510ce1f83f3a0602747a2b", "config": 2},
+                   "sha1": "8ba9e4cc6b94f12503614d6c61024e55f9f8813a", "config": 2},
     "all depthwise kernels": {"bytes_per_launch": 13.20e6, "source": "paper_2103_16827_b200/csrc/dw_tc.cu",
-                              "sha1": "ca47bb3d387106f1e8510ce1f83f3a0602747a2b", "config": 2},
+                              "sha1": "8ba9e4cc6b94f12503614d6c61024e55f9f8813a", "config": 2},
 }
 
 
