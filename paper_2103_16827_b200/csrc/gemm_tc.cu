@@ -34,8 +34,11 @@ constexpr int BM = 128;            // output channels per MMA tile (TMEM lanes)
 constexpr int MAX_W_STAGES = 8;    // weight ring: as many stages as shared memory leaves room for
 constexpr int MAX_KB = 16;         // C_in <= 1024
 static_assert(MAX_KB + MAX_W_STAGES + 2 <= 31, "the barriers are initialised by one warp, one lane each");
-constexpr int EPI_PARTS = 4;        // epilogue warps per 32-channel quarter (they split the frames)
-constexpr int EPI_WARPS = 4 * EPI_PARTS;
+// Sixteen epilogue warps. As one group, four per 32-channel quarter split a tile's frames; as two groups of eight
+// (template parameter GROUPS = 2), group g takes the output tiles of accumulator buffer g and two warps per
+// quarter split the frames, so that the fixed part of one tile's epilogue (constants, waits, store issue)
+// overlaps the arithmetic of the other tile's.
+constexpr int EPI_WARPS = 16;
 constexpr int THREADS = 64 + 32 * EPI_WARPS;
 constexpr int ACC_STRIDE = 256;    // TMEM columns between the two accumulator buffers
 constexpr int TMEM_COLS = 512;
@@ -48,7 +51,7 @@ struct GemmParams {
     int n_items;
     int w_stages;                  // depth of the weight ring (<= MAX_W_STAGES)
     int out_bytes;                 // bytes of the output staging area (one block per epilogue warp)
-    int stage_w;                   // bytes per staged row of the wider warps (16 * ceil(chunks / EPI_PARTS))
+    int stage_w;                   // bytes per staged row of the wider warps (16 * ceil(chunks / warps per quarter))
     const int32_t* bias;
     const int32_t* mult;
     const uint8_t* shift;
@@ -79,7 +82,7 @@ __device__ __forceinline__ void item_coords(const GemmParams& p, int item, int& 
     m_hi = min(p.m_tiles, m_lo + per);
 }
 
-template <int BK>
+template <int BK, int GROUPS>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                   const __grid_constant__ CUtensorMap tmXl,
@@ -96,6 +99,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     uint8_t* Os = Ws + W_STAGES * W_STAGE_BYTES;                // [128 channels][BN frames] output staging
     SharedTail* sh = (SharedTail*)(Os + p.out_bytes);
 
+    constexpr int EPI_PARTS = EPI_WARPS / (4 * GROUPS);     // warps per quarter that share one tile
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     // one barrier (pair) per thread of warp 2, so that the set-up is not one thread's serial chain
@@ -108,7 +112,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             ptx::mbar_init(ptx::smem_u32(&sh->wempty[lane - MAX_KB]), 1);
         } else if (lane < MAX_KB + MAX_W_STAGES + 2) {
             ptx::mbar_init(ptx::smem_u32(&sh->accfull[lane - MAX_KB - MAX_W_STAGES]), 1);
-            ptx::mbar_init(ptx::smem_u32(&sh->accempty[lane - MAX_KB - MAX_W_STAGES]), EPI_WARPS);
+            ptx::mbar_init(ptx::smem_u32(&sh->accempty[lane - MAX_KB - MAX_W_STAGES]), EPI_WARPS / GROUPS);
         }
         if (lane == 31) sh->abort_flag = 0;
         ptx::mbar_fence_init();
@@ -261,7 +265,8 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     } else {
         // ------------------------------------------------------------------ epilogue warps
         const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31 belong to this warp
-        const int part = (warp - 2) >> 2;             // which share of the tile's 16-frame chunks
+        const int part = ((warp - 2) >> 2) % EPI_PARTS;   // which share of the tile's 16-frame chunks
+        const int egrp = (warp - 2) / (4 * EPI_PARTS);     // which accumulator buffer's tiles (GROUPS == 2)
         const int n_chunks = p.BN >> 4;
         const int c_lo = part * n_chunks / EPI_PARTS;
         const int c_hi = (part + 1) * n_chunks / EPI_PARTS;
@@ -280,6 +285,7 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             for (int mi = 0; mi < mc && ok; ++mi, ++acount) {
                 const int m = m_lo + (mi + (int)(blockIdx.x % mc)) % mc;   // the order the producer and MMA warps use
                 const int a = acount & 1u;
+                if (GROUPS == 2 && a != egrp) continue;         // the other group's tile
                 EpiThread e;
                 const int o = m * BM + quarter * 32 + lane;
                 e.valid_o = o < p.C_out;
@@ -406,9 +412,10 @@ bool qasr_encode_map_u8(qasr_ctx* ctx, CUtensorMap* map, const void* base, int r
 static const size_t kSmemLimit = 227 * 1024;
 
 int qasr_gemm_tc_init(qasr_ctx* ctx) {
-    cudaError_t e = cudaFuncSetAttribute(qasr::tc::gemm_i8_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(qasr::tc::gemm_i8_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
+    cudaError_t e = cudaFuncSetAttribute(qasr::tc::gemm_i8_tc_kernel<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(qasr::tc::gemm_i8_tc_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(qasr::tc::gemm_i8_tc_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(qasr::tc::gemm_i8_tc_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
     if (e != cudaSuccess) {
         snprintf(ctx->err, sizeof(ctx->err), "cudaFuncSetAttribute(gemm_i8_tc_kernel) failed: %s", cudaGetErrorString(e));
         return QASR_ERR_CUDA;
@@ -462,11 +469,28 @@ int qasr_launch_gemm_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
     // pipeline block, staging tile and weight-ring depth from what shared memory allows
     const int BK = a.C_in % 128 == 0 ? 128 : 64;
     const int n_chunks = p.BN / 16;
-    p.stage_w = 16 * ((n_chunks + EPI_PARTS - 1) / EPI_PARTS);
-    p.out_bytes = a.y ? (EPI_WARPS * 32 * p.stage_w + 1023) / 1024 * 1024 : 0;
+    // Two epilogue groups pay where a CTA has at least two output tiles per item and the wider staging blocks
+    // still leave a weight ring of four stages (C_in <= 256), or where an item has so many output tiles that the
+    // ring's depth no longer matters (measured at B=32: 256->256 7.8 -> 7.5 us, 256->512 11.8 -> 11.1 us,
+    // 512->1024 26.4 -> 24.3 us; 512->512 with its four tiles and a two-stage ring: 13.1 -> 13.3 us, one group kept).
+    const int per_item = (p.m_tiles + p.m_groups - 1) / p.m_groups;
+    auto layout = [&](int groups, int& stage_w, int& out_bytes, int& w_stages) {
+        const int parts = EPI_WARPS / (4 * groups);
+        stage_w = 16 * ((n_chunks + parts - 1) / parts);
+        out_bytes = a.y ? (EPI_WARPS * 32 * stage_w + 1023) / 1024 * 1024 : 0;
+        const size_t fixed_ = 1024 + (size_t)a.C_in * p.NC * 128 + out_bytes + sizeof(SharedTail);
+        w_stages = fixed_ >= kSmemLimit ? 0 : (int)((kSmemLimit - fixed_) / (size_t)(BM * BK));
+        if (w_stages > MAX_W_STAGES) w_stages = MAX_W_STAGES;
+    };
+    int GROUPS = 1;
+    {
+        int sw, ob, ws;
+        layout(2, sw, ob, ws);
+        if (a.y && per_item >= 2 && ws >= 2 && (ws >= 4 || per_item >= 6)) GROUPS = 2;
+    }
+    const int EPI_PARTS = EPI_WARPS / (4 * GROUPS);
+    layout(GROUPS, p.stage_w, p.out_bytes, p.w_stages);
     const size_t fixed = 1024 + (size_t)a.C_in * p.NC * 128 + p.out_bytes + sizeof(SharedTail);
-    p.w_stages = (int)((kSmemLimit - fixed) / (size_t)(BM * BK));
-    if (p.w_stages > MAX_W_STAGES) p.w_stages = MAX_W_STAGES;
     if (p.w_stages < 2) return QASR_ERR_SHAPE;
     CUtensorMap tmW, tmX, tmXl, tmY, tmYw;
     {
@@ -501,8 +525,10 @@ int qasr_launch_gemm_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
     const int grid = p.n_items < qasr_grid_slots(ctx) ? p.n_items : qasr_grid_slots(ctx);
     QasrLaunchScope ls(ctx, QASR_K_GEMM_TC, qasr_conv_macs(a), qasr_conv_bytes(a));
     cudaError_t e = BK == 128
-        ? qasr_launch_overlapped(ctx, gemm_i8_tc_kernel<128>, dim3(grid), dim3(THREADS), smem, tmW, tmX, tmXl, tmY, tmYw, p)
-        : qasr_launch_overlapped(ctx, gemm_i8_tc_kernel<64>, dim3(grid), dim3(THREADS), smem, tmW, tmX, tmXl, tmY, tmYw, p);
+        ? (GROUPS == 2 ? qasr_launch_overlapped(ctx, gemm_i8_tc_kernel<128, 2>, dim3(grid), dim3(THREADS), smem, tmW, tmX, tmXl, tmY, tmYw, p)
+                       : qasr_launch_overlapped(ctx, gemm_i8_tc_kernel<128, 1>, dim3(grid), dim3(THREADS), smem, tmW, tmX, tmXl, tmY, tmYw, p))
+        : (GROUPS == 2 ? qasr_launch_overlapped(ctx, gemm_i8_tc_kernel<64, 2>, dim3(grid), dim3(THREADS), smem, tmW, tmX, tmXl, tmY, tmYw, p)
+                       : qasr_launch_overlapped(ctx, gemm_i8_tc_kernel<64, 1>, dim3(grid), dim3(THREADS), smem, tmW, tmX, tmXl, tmY, tmYw, p));
     if (e != cudaSuccess) {
         snprintf(ctx->err, sizeof(ctx->err), "gemm_i8_tc_kernel launch failed: %s", cudaGetErrorString(e));
         return QASR_ERR_CUDA;
