@@ -469,10 +469,11 @@ int qasr_launch_gemm_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
     // pipeline block, staging tile and weight-ring depth from what shared memory allows
     const int BK = a.C_in % 128 == 0 ? 128 : 64;
     const int n_chunks = p.BN / 16;
-    // Two epilogue groups pay where a CTA has at least two output tiles per item and the wider staging blocks
-    // still leave a weight ring of four stages (C_in <= 256), or where an item has so many output tiles that the
-    // ring's depth no longer matters (measured at B=32: 256->256 7.8 -> 7.5 us, 256->512 11.8 -> 11.1 us,
-    // 512->1024 26.4 -> 24.3 us; 512->512 with its four tiles and a two-stage ring: 13.1 -> 13.3 us, one group kept).
+    // Two epilogue groups pay where a CTA works through at least two output tiles (of one item or of several) and the
+    // wider staging blocks still leave a weight ring of four stages, or where its items have one output tile each, so
+    // that every tile waits for a new activation tile and the ring's depth does not matter (measured at B=32:
+    // 256->256 7.8 -> 7.5 us, 256->512 11.8 -> 11.1 us, 256->1024 20.2 -> 18.1 us, 512->1024 26.5 -> 24.4 us;
+    // 512->512, four tiles per item and a two-stage ring: 13.1 -> 13.3 us, at B=256 75.7 -> 80.8 us, one group kept).
     const int per_item = (p.m_tiles + p.m_groups - 1) / p.m_groups;
     auto layout = [&](int groups, int& stage_w, int& out_bytes, int& w_stages) {
         const int parts = EPI_WARPS / (4 * groups);
@@ -486,7 +487,9 @@ int qasr_launch_gemm_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
     {
         int sw, ob, ws;
         layout(2, sw, ob, ws);
-        if (a.y && per_item >= 2 && ws >= 2 && (ws >= 4 || per_item >= 6)) GROUPS = 2;
+        const int slots = p.n_items < qasr_grid_slots(ctx) ? p.n_items : qasr_grid_slots(ctx);
+        const int tiles_per_cta = (p.n_items + slots - 1) / slots * per_item;
+        if (a.y && tiles_per_cta >= 2 && ws >= 2 && (ws >= 4 || (per_item == 1 && tiles_per_cta >= 6))) GROUPS = 2;
     }
     const int EPI_PARTS = EPI_WARPS / (4 * GROUPS);
     layout(GROUPS, p.stage_w, p.out_bytes, p.w_stages);
