@@ -106,11 +106,9 @@ __device__ __forceinline__ int4 requant16_dw(const uint32_t (&r)[16], int mn, lo
     int q[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
-        long long p64;
-        asm("mad.wide.s32 %0, %1, %2, %3;" : "=l"(p64) : "r"((int)r[i]), "r"(mn), "l"(half64));
-        if (MODE == 0) q[i] = (int)(p64 >> 32);
-        else if (MODE == 1) q[i] = (int)(p64 >> 32) >> (sn - 32);
-        else q[i] = (int)clamp_i8_ll(p64 >> sn);
+        if (MODE == 0) q[i] = ptx::mad_hi64((int)r[i], mn, half64);
+        else if (MODE == 1) q[i] = ptx::mad_hi64((int)r[i], mn, half64) >> (sn - 32);
+        else q[i] = (int)clamp_i8_ll(((long long)(int)r[i] * (long long)mn + half64) >> sn);
     }
     int4 out;
     out.x = (int)ptx::pack4_sat_s8(q[0], q[1], q[2], q[3]);

@@ -195,5 +195,21 @@ __device__ __forceinline__ uint32_t pack4_sat_s8(int v0, int v1, int v2, int v3)
     return pack_sat_s8(v1, v0, pack_sat_s8(v3, v2, 0u));
 }
 
+// High word of the 64-bit sum a * b + c. Written as a carry chain of the two 32-bit halves, which the assembler
+// turns into one multiply-add that takes the 64-bit addend; `mad.wide.s32` with a 64-bit addend comes out as a
+// wide multiply followed by a two-instruction 64-bit add (counted per opcode on a B200: 3 instead of 1 per value).
+__device__ __forceinline__ int mad_hi64(int a, int b, long long c) {
+    int lo, hi;
+    asm("{mad.lo.cc.s32 %0, %2, %3, %4;\n\tmadc.hi.s32 %1, %2, %3, %5;}"
+        : "=r"(lo), "=r"(hi) : "r"(a), "r"(b), "r"((int)c), "r"((int)(c >> 32)));
+    return hi;
+}
+// max(byte, 0) on four packed int8: the sign of every byte replicated over the byte, then cleared.
+__device__ __forceinline__ uint32_t relu4_s8(uint32_t w) {
+    uint32_t sign;
+    asm("prmt.b32 %0, %1, 0, 0xba98;" : "=r"(sign) : "r"(w));
+    return w & ~sign;
+}
+
 }  // namespace ptx
 }  // namespace qasr

@@ -47,19 +47,21 @@ __device__ __forceinline__ int4 requant16(const uint32_t (&r)[16], const Channel
     const int sh = rq.s - 32;
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
-        long long p64;
-        asm("mad.wide.s32 %0, %1, %2, %3;" : "=l"(p64) : "r"((int)r[i]), "r"(rq.m), "l"(rq.c64));
-        int v = (int)(p64 >> 32);
+        int v = ptx::mad_hi64((int)r[i], rq.m, rq.c64);
         if (MODE == 1) v >>= sh;
-        if (RELU) v = max(v, 0);
         q[i] = v;
     }
-    int4 out;
-    out.x = (int)ptx::pack4_sat_s8(q[0], q[1], q[2], q[3]);
-    out.y = (int)ptx::pack4_sat_s8(q[4], q[5], q[6], q[7]);
-    out.z = (int)ptx::pack4_sat_s8(q[8], q[9], q[10], q[11]);
-    out.w = (int)ptx::pack4_sat_s8(q[12], q[13], q[14], q[15]);
-    return out;
+    // saturate to int8 first, then ReLU on the packed bytes: max(sat8(v), 0) = sat8(max(v, 0))
+    uint4 out;
+    out.x = ptx::pack4_sat_s8(q[0], q[1], q[2], q[3]);
+    out.y = ptx::pack4_sat_s8(q[4], q[5], q[6], q[7]);
+    out.z = ptx::pack4_sat_s8(q[8], q[9], q[10], q[11]);
+    out.w = ptx::pack4_sat_s8(q[12], q[13], q[14], q[15]);
+    if (RELU) {
+        out.x = ptx::relu4_s8(out.x); out.y = ptx::relu4_s8(out.y);
+        out.z = ptx::relu4_s8(out.z); out.w = ptx::relu4_s8(out.w);
+    }
+    return make_int4((int)out.x, (int)out.y, (int)out.z, (int)out.w);
 }
 
 // Everything an epilogue thread needs to turn 16 accumulator columns into 16 output bytes.
