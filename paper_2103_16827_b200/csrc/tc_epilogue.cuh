@@ -108,7 +108,17 @@ __device__ __forceinline__ int4 epilogue16(const Params& p, const EpiThread& e, 
                 }
             }
 #pragma unroll
-            for (int i = 0; i < 16; ++i) q[i] = p.relu ? max(v[i], 0) : v[i];
+            for (int i = 0; i < 16; ++i) q[i] = v[i];
+            uint4 o;
+            o.x = ptx::pack4_sat_s8(q[0], q[1], q[2], q[3]);
+            o.y = ptx::pack4_sat_s8(q[4], q[5], q[6], q[7]);
+            o.z = ptx::pack4_sat_s8(q[8], q[9], q[10], q[11]);
+            o.w = ptx::pack4_sat_s8(q[12], q[13], q[14], q[15]);
+            if (p.relu) {       // on the packed bytes: max(sat8(v), 0) = sat8(max(v, 0))
+                o.x = ptx::relu4_s8(o.x); o.y = ptx::relu4_s8(o.y);
+                o.z = ptx::relu4_s8(o.z); o.w = ptx::relu4_s8(o.w);
+            }
+            return make_int4((int)o.x, (int)o.y, (int)o.z, (int)o.w);
         } else {
             long long v[16];
 #pragma unroll
