@@ -198,15 +198,25 @@ ELEMENTWISE_KERNELS = ("residual_add", "glu", "dequant", "conv_tc_prepare")
 # on `microbench conv 32 512 512 800` and `microbench dw 32 512 800 75`). ncu flushes the caches before every
 # captured launch, so this is cold-cache traffic: the input tensor read once, the output still in L2 when the
 # kernel ends; inside the step the input is L2-resident as well and DRAM sees about 1 MB per launch. Recorded
-# with the SHA-1 of the kernel source they were taken on: a changed kernel reports null.
+# with the SHA-1 of the kernel sources they were taken on: a changed kernel reports null.
 TRAFFIC = {
-    "gemm_i8_tc": {"bytes_per_launch": 13.52e6, "source": "paper_2103_16827_b200/csrc/gemm_tc.cu",
-                   "sha1": "997be66518dcc5bc52cbc10c5f332fb04e494dc2", "config": 2},
-    "dw_conv_tc": {"bytes_per_launch": 13.20e6, "source": "paper_2103_16827_b200/csrc/dw_tc.cu",
-                   "sha1": "8ba9e4cc6b94f12503614d6c61024e55f9f8813a", "config": 2},
-    "all depthwise kernels": {"bytes_per_launch": 13.20e6, "source": "paper_2103_16827_b200/csrc/dw_tc.cu",
-                              "sha1": "8ba9e4cc6b94f12503614d6c61024e55f9f8813a", "config": 2},
+    "gemm_i8_tc": {"bytes_per_launch": 13.52e6, "sources": ["gemm_tc.cu", "tc_epilogue.cuh", "sm100_ptx.cuh"],
+                   "sha1": "78f9bda46f966b944aca2b3c59f743e3ad8d911f", "config": 2},
+    "dw_conv_tc": {"bytes_per_launch": 13.20e6, "sources": ["dw_tc.cu", "sm100_ptx.cuh"],
+                   "sha1": "b99cddb39aeadef1682cdee04fbbc4fe2dbe5387", "config": 2},
+    "all depthwise kernels": {"bytes_per_launch": 13.20e6, "sources": ["dw_tc.cu", "sm100_ptx.cuh"],
+                              "sha1": "b99cddb39aeadef1682cdee04fbbc4fe2dbe5387", "config": 2},
 }
+
+
+def sources_sha1(names):
+    """SHA-1 over the named kernel sources (files of the package's csrc folder), in the order given."""
+    import hashlib
+    h = hashlib.sha1()
+    for n in names:
+        with open(os.path.join(ROOT, "paper_2103_16827_b200", "csrc", n), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
 
 
 def max_over_ranks(ms, world, device):
@@ -226,14 +236,12 @@ def job_throughput(world, frames_per_rank_step, steps, total_ms):
 
 
 def recorded_traffic(kernel, config):
-    import hashlib
     rec = TRAFFIC.get(kernel)
     if not rec or rec["config"] != config:
         return None
     try:
-        with open(os.path.join(ROOT, rec["source"]), "rb") as f:
-            if hashlib.sha1(f.read()).hexdigest() != rec["sha1"]:
-                return None
+        if sources_sha1(rec["sources"]) != rec["sha1"]:
+            return None
     except OSError:
         return None
     return rec["bytes_per_launch"]
