@@ -82,7 +82,7 @@ __device__ __forceinline__ void item_coords(const GemmParams& p, int item, int& 
     m_hi = min(p.m_tiles, m_lo + per);
 }
 
-template <int BK, int GROUPS>
+template <int BK, int GROUPS, bool RES1>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                   const __grid_constant__ CUtensorMap tmXl,
@@ -302,8 +302,19 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                 e.all_fast = __all_sync(0xffffffffu, e.rq.fast != 0);
                 const bool all_s32 = __all_sync(0xffffffffu, e.rq.s == 32);
                 e.row = ((size_t)b * p.C_out + (e.valid_o ? o : 0)) * p.T;
-                // 0: shift == 32 in every lane, 1: shift >= 32, 2: anything (also residual terms)
-                const int mode = p.terms.n > 0 ? 2 : (all_s32 ? 0 : (e.all_fast ? 1 : 2));
+                // 0: shift == 32 in every lane, 1: shift >= 32, 2: anything (also residual terms),
+                // 3: one residual tensor, 32-bit products, shift >= 32 (its words are fetched a chunk ahead)
+                const int mode = RES1 && e.all_fast ? 3
+                                 : p.terms.n > 0 ? 2 : (all_s32 ? 0 : (e.all_fast ? 1 : 2));
+                ResidualOne ro;
+                const int4* res_row = nullptr;      // this thread's residual words for chunk c at res_row[c]
+                int4 res_next = make_int4(0, 0, 0, 0);
+                if (RES1 && mode == 3) {
+                    ro.m0 = p.terms.mult[0]; ro.s0 = p.terms.shift[0]; ro.h0 = 1 << (ro.s0 - 1);
+                    ro.m1 = p.terms.mult[1]; ro.s1 = p.terms.shift[1]; ro.h1 = 1 << (ro.s1 - 1);
+                    res_row = reinterpret_cast<const int4*>(p.terms.ptr[1] + e.row + t0);
+                    if (e.valid_o && c_lo < c_hi && t0 + c_lo * 16 < p.T) res_next = __ldg(res_row + c_lo);
+                }
                 if (!p.y32) {
                     // this warp's previous TMA store must have finished reading its staging block
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -337,6 +348,11 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                         out = p.relu ? requant16<0, true>(r, e.rq) : requant16<0, false>(r, e.rq);
                     } else if (mode == 1) {
                         out = p.relu ? requant16<1, true>(r, e.rq) : requant16<1, false>(r, e.rq);
+                    } else if (RES1 && mode == 3) {
+                        const int4 res = res_next;
+                        if (e.valid_o && c + 1 < c_hi && t0 + (c + 1) * 16 < p.T) res_next = __ldg(res_row + c + 1);
+                        else res_next = make_int4(0, 0, 0, 0);
+                        out = p.relu ? epilogue16_res1<true>(r, e.rq, res, ro) : epilogue16_res1<false>(r, e.rq, res, ro);
                     } else {
                         const int t = t0 + c * 16;
                         out = epilogue16(p, e, r, t, e.valid_o && t < p.T);
@@ -412,10 +428,14 @@ bool qasr_encode_map_u8(qasr_ctx* ctx, CUtensorMap* map, const void* base, int r
 static const size_t kSmemLimit = 227 * 1024;
 
 int qasr_gemm_tc_init(qasr_ctx* ctx) {
-    cudaError_t e = cudaFuncSetAttribute(qasr::tc::gemm_i8_tc_kernel<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(qasr::tc::gemm_i8_tc_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(qasr::tc::gemm_i8_tc_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(qasr::tc::gemm_i8_tc_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
+    cudaError_t e = cudaSuccess;
+    auto allow = [&](auto kernel) {
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
+    };
+    allow(qasr::tc::gemm_i8_tc_kernel<64, 1, false>); allow(qasr::tc::gemm_i8_tc_kernel<64, 2, false>);
+    allow(qasr::tc::gemm_i8_tc_kernel<128, 1, false>); allow(qasr::tc::gemm_i8_tc_kernel<128, 2, false>);
+    allow(qasr::tc::gemm_i8_tc_kernel<64, 1, true>); allow(qasr::tc::gemm_i8_tc_kernel<64, 2, true>);
+    allow(qasr::tc::gemm_i8_tc_kernel<128, 1, true>); allow(qasr::tc::gemm_i8_tc_kernel<128, 2, true>);
     if (e != cudaSuccess) {
         snprintf(ctx->err, sizeof(ctx->err), "cudaFuncSetAttribute(gemm_i8_tc_kernel) failed: %s", cudaGetErrorString(e));
         return QASR_ERR_CUDA;
@@ -527,11 +547,20 @@ int qasr_launch_gemm_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
     const size_t smem = fixed + (size_t)p.w_stages * BM * BK;
     const int grid = p.n_items < qasr_grid_slots(ctx) ? p.n_items : qasr_grid_slots(ctx);
     QasrLaunchScope ls(ctx, QASR_K_GEMM_TC, qasr_conv_macs(a), qasr_conv_bytes(a));
-    cudaError_t e = BK == 128
-        ? (GROUPS == 2 ? qasr_launch_overlapped(ctx, gemm_i8_tc_kernel<128, 2>, dim3(grid), dim3(THREADS), smem, tmW, tmX, tmXl, tmY, tmYw, p)
-                       : qasr_launch_overlapped(ctx, gemm_i8_tc_kernel<128, 1>, dim3(grid), dim3(THREADS), smem, tmW, tmX, tmXl, tmY, tmYw, p))
-        : (GROUPS == 2 ? qasr_launch_overlapped(ctx, gemm_i8_tc_kernel<64, 2>, dim3(grid), dim3(THREADS), smem, tmW, tmX, tmXl, tmY, tmYw, p)
-                       : qasr_launch_overlapped(ctx, gemm_i8_tc_kernel<64, 1>, dim3(grid), dim3(THREADS), smem, tmW, tmX, tmXl, tmY, tmYw, p));
+    // the residual instantiation: one residual tensor beside the layer's own output, constants that keep every
+    // product inside 32 bits (a block's last layer); everything else runs the kernel without that code
+    const bool res1 = a.y && a.terms.n == 2 && p.terms_fast;
+    auto launch = [&](auto kernel) {
+        return qasr_launch_overlapped(ctx, kernel, dim3(grid), dim3(THREADS), smem, tmW, tmX, tmXl, tmY, tmYw, p);
+    };
+    cudaError_t e;
+    if (BK == 128) {
+        if (GROUPS == 2) e = res1 ? launch(gemm_i8_tc_kernel<128, 2, true>) : launch(gemm_i8_tc_kernel<128, 2, false>);
+        else e = res1 ? launch(gemm_i8_tc_kernel<128, 1, true>) : launch(gemm_i8_tc_kernel<128, 1, false>);
+    } else {
+        if (GROUPS == 2) e = res1 ? launch(gemm_i8_tc_kernel<64, 2, true>) : launch(gemm_i8_tc_kernel<64, 2, false>);
+        else e = res1 ? launch(gemm_i8_tc_kernel<64, 1, true>) : launch(gemm_i8_tc_kernel<64, 1, false>);
+    }
     if (e != cudaSuccess) {
         snprintf(ctx->err, sizeof(ctx->err), "gemm_i8_tc_kernel launch failed: %s", cudaGetErrorString(e));
         return QASR_ERR_CUDA;

@@ -64,6 +64,46 @@ __device__ __forceinline__ int4 requant16(const uint32_t (&r)[16], const Channel
     return make_int4((int)out.x, (int)out.y, (int)out.z, (int)out.w);
 }
 
+// The epilogue of a block's last layer in its common form: one residual tensor beside the layer's own output, every
+// constant small enough for 32-bit products (the caller has checked both, and that every lane's shift is >= 32).
+// `res` holds the residual's 16 int8 of this thread's channel, fetched a chunk ahead by the caller.
+//   a = sat8(RS((acc + bias) * m, s));  v = RS(a * m0, s0) + RS(r * m1, s1);  y = sat8(relu?(v))
+struct ResidualOne {
+    int m0, s0, h0;    // the layer's own output: multiplier, shift, 2^(shift-1)
+    int m1, s1, h1;    // the residual tensor
+};
+// Byte B of a word, sign-extended: one prmt whose selector replicates the byte's sign over the upper three bytes.
+template <int B>
+__device__ __forceinline__ int sext_byte(uint32_t w) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, 0, %2;" : "=r"(d) : "r"(w), "n"(B | ((8 | B) << 4) | ((8 | B) << 8) | ((8 | B) << 12)));
+    return (int)d;
+}
+template <bool RELU>
+__device__ __forceinline__ int4 epilogue16_res1(const uint32_t (&r)[16], const ChannelRq& rq, const int4& res,
+                                                const ResidualOne& t) {
+    const int sh = rq.s - 32;
+    const uint32_t words[4] = {(uint32_t)res.x, (uint32_t)res.y, (uint32_t)res.z, (uint32_t)res.w};
+    int q[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const int a = clamp_i8(ptx::mad_hi64((int)r[i], rq.m, rq.c64) >> sh);
+        const uint32_t w = words[i >> 2];
+        const int rb = (i & 3) == 0 ? sext_byte<0>(w) : (i & 3) == 1 ? sext_byte<1>(w) : (i & 3) == 2 ? sext_byte<2>(w) : sext_byte<3>(w);
+        q[i] = ((a * t.m0 + t.h0) >> t.s0) + ((rb * t.m1 + t.h1) >> t.s1);
+    }
+    uint4 o;
+    o.x = ptx::pack4_sat_s8(q[0], q[1], q[2], q[3]);
+    o.y = ptx::pack4_sat_s8(q[4], q[5], q[6], q[7]);
+    o.z = ptx::pack4_sat_s8(q[8], q[9], q[10], q[11]);
+    o.w = ptx::pack4_sat_s8(q[12], q[13], q[14], q[15]);
+    if (RELU) {       // on the packed bytes: max(sat8(v), 0) = sat8(max(v, 0))
+        o.x = ptx::relu4_s8(o.x); o.y = ptx::relu4_s8(o.y);
+        o.z = ptx::relu4_s8(o.z); o.w = ptx::relu4_s8(o.w);
+    }
+    return make_int4((int)o.x, (int)o.y, (int)o.z, (int)o.w);
+}
+
 // Everything an epilogue thread needs to turn 16 accumulator columns into 16 output bytes.
 struct EpiThread {
     ChannelRq rq;

@@ -36,6 +36,8 @@ def main():
     ap.add_argument("--shift", type=int, default=24)
     ap.add_argument("--no-scratch", action="store_true", help="conv: lend no scratch (K-tap convolutions then use the generic kernel)")
     ap.add_argument("--no-delay", action="store_true", help="do not queue the launches behind a device delay")
+    ap.add_argument("--residual", type=int, default=0,
+                    help="conv: number of residual tensors added in the epilogue (each rescaled on its own)")
     args = ap.parse_args()
     rng = np.random.Generator(np.random.PCG64(0))
     ctx = Context(0)
@@ -62,8 +64,15 @@ def main():
         if not args.no_scratch:
             ctx.set_conv_scratch(torch.empty(max(256, ctx.conv_scratch_bytes(B, Ci, Co, T, K, args.stride)),
                                              dtype=torch.uint8, device="cuda"))
-        fn = lambda: ctx.conv(x, w, bias, 4096, m, s, True, stride=args.stride, dilation=args.dilation, y=y)
-        macs, nbytes = B * Ci * Co * T_out * K, B * (T * Ci + T_out * Co) + Ci * Co * K
+        res = [_dev(rng.integers(-128, 128, size=(B, Co, T_out), dtype=np.int8)) for _ in range(args.residual)]
+        tm = [int(v) for v in rng.integers(1 << 13, 1 << 14, size=args.residual + 1)]
+        ts = [15] * (args.residual + 1)
+        if args.residual:
+            fn = lambda: ctx.conv(x, w, bias, 4096, m, s, True, stride=args.stride, dilation=args.dilation,
+                                  terms=[None] + res, term_mult=tm, term_shift=ts, y=y)
+        else:
+            fn = lambda: ctx.conv(x, w, bias, 4096, m, s, True, stride=args.stride, dilation=args.dilation, y=y)
+        macs, nbytes = B * Ci * Co * T_out * K, B * (T * Ci + T_out * Co * (1 + args.residual)) + Ci * Co * K
     elif args.op == "dw":
         B, C, T, K = args.dims
         x = _dev(rng.integers(-128, 128, size=(B, C, T), dtype=np.int8))
