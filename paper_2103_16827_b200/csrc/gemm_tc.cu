@@ -352,7 +352,8 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                         const int4 res = res_next;
                         if (e.valid_o && c + 1 < c_hi && t0 + (c + 1) * 16 < p.T) res_next = __ldg(res_row + c + 1);
                         else res_next = make_int4(0, 0, 0, 0);
-                        out = p.relu ? epilogue16_res1<true>(r, e.rq, res, ro) : epilogue16_res1<false>(r, e.rq, res, ro);
+                        if (all_s32) out = p.relu ? epilogue16_res1<true, true>(r, e.rq, res, ro) : epilogue16_res1<false, true>(r, e.rq, res, ro);
+                        else out = p.relu ? epilogue16_res1<true, false>(r, e.rq, res, ro) : epilogue16_res1<false, false>(r, e.rq, res, ro);
                     } else {
                         const int t = t0 + c * 16;
                         out = epilogue16(p, e, r, t, e.valid_o && t < p.T);
