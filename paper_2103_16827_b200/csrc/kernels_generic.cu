@@ -2,6 +2,7 @@
 // tensor-core and vectorised kernels do not take (odd sizes, stride/dilation 2, tiny channel
 // counts) and for the element-wise steps (residual add, final dequantisation).
 #include "qasr_device.cuh"
+#include "sm100_ptx.cuh"
 
 namespace qasr {
 
@@ -217,6 +218,24 @@ glu_kernel(const int8_t* x, int C, int T, size_t n, int q_c, const int32_t* mult
 }
 
 // The same gate, 16 consecutive frames of one channel per thread (16-byte loads and stores); T16 = T / 16.
+// The channel's dyadic constant is normalised to a shift of at least 32 where the multiplier has the head-room
+// ((m << k, s + k) is the same number), so that the rescaling is the high word of one multiply-add.
+template <int W>
+__device__ __forceinline__ void glu_word(uint32_t aw, uint32_t gw, int q_c, int full, int mn, long long half, int sn,
+                                         bool fast, int (&q)[16]) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int a = e == 0 ? ptx::sext_byte<0>(aw) : e == 1 ? ptx::sext_byte<1>(aw) : e == 2 ? ptx::sext_byte<2>(aw) : ptx::sext_byte<3>(aw);
+        const int g = e == 0 ? ptx::sext_byte<0>(gw) : e == 1 ? ptx::sext_byte<1>(gw) : e == 2 ? ptx::sext_byte<2>(gw) : ptx::sext_byte<3>(gw);
+        const int pq = q_c - min(abs(g), q_c);
+        const int h = full - pq * pq;
+        const int sig = g >= 0 ? h : full - h;
+        const int v = a * sig;                          // |v| <= 128 * 2 * 128^2 < 2^23
+        q[4 * W + e] = fast ? ptx::mad_hi64(v, mn, half) >> (sn - 32)
+                            : (int)clamp_i8_ll(((long long)v * (long long)mn + half) >> sn);
+    }
+}
+
 __global__ void __launch_bounds__(256)
 glu_vec16_kernel(const int8_t* __restrict__ x, int C, int T16, unsigned items, int q_c, const int32_t* mult,
                  const uint8_t* shift, int8_t* __restrict__ y, unsigned* status) {
@@ -224,31 +243,29 @@ glu_vec16_kernel(const int8_t* __restrict__ x, int C, int T16, unsigned items, i
     if (i >= items) return;
     const unsigned t16 = i % (unsigned)T16, bc = i / (unsigned)T16;
     const unsigned c = bc % (unsigned)C, b = bc / (unsigned)C;
-    int m, s;
-    load_rq(mult, shift, (int)c, m, s, status);
     const size_t row = (size_t)T16 * 16;
     const size_t ia = ((size_t)b * 2 * C + c) * row + (size_t)t16 * 16;
     const int4 av = __ldg(reinterpret_cast<const int4*>(x + ia));
     const int4 gv = __ldg(reinterpret_cast<const int4*>(x + ia + (size_t)C * row));
-    const int aw[4] = {av.x, av.y, av.z, av.w}, gw[4] = {gv.x, gv.y, gv.z, gv.w};
+    int m, s;
+    load_rq(mult, shift, (int)c, m, s, status);
+    const int kmax = min(__clz(m) - 1, 62 - s);
+    const int k = (s <= 32 && 32 - s <= kmax) ? 32 - s : max(kmax, 0);
+    const int mn = m << k, sn = s + k;
+    const long long half = 1LL << (sn - 1);
+    const bool fast = sn >= 32;
     const int full = 2 * q_c * q_c;
-    const long long half = 1LL << (s - 1);
-    int ow[4];
-#pragma unroll
-    for (int wd = 0; wd < 4; ++wd) {
-        int q[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int a = (int)(int8_t)(aw[wd] >> (8 * e));
-            const int g = (int)(int8_t)(gw[wd] >> (8 * e));
-            const int pq = q_c - min(abs(g), q_c);
-            const int h = full - pq * pq;
-            const int sig = g >= 0 ? h : full - h;
-            q[e] = (int)clamp_i8_ll(((long long)(a * sig) * (long long)m + half) >> s);
-        }
-        ow[wd] = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | ((q[3] & 0xff) << 24);
-    }
-    *reinterpret_cast<int4*>(y + ((size_t)bc * row + (size_t)t16 * 16)) = make_int4(ow[0], ow[1], ow[2], ow[3]);
+    int q[16];
+    glu_word<0>((uint32_t)av.x, (uint32_t)gv.x, q_c, full, mn, half, sn, fast, q);
+    glu_word<1>((uint32_t)av.y, (uint32_t)gv.y, q_c, full, mn, half, sn, fast, q);
+    glu_word<2>((uint32_t)av.z, (uint32_t)gv.z, q_c, full, mn, half, sn, fast, q);
+    glu_word<3>((uint32_t)av.w, (uint32_t)gv.w, q_c, full, mn, half, sn, fast, q);
+    int4 out;
+    out.x = (int)ptx::pack4_sat_s8(q[0], q[1], q[2], q[3]);
+    out.y = (int)ptx::pack4_sat_s8(q[4], q[5], q[6], q[7]);
+    out.z = (int)ptx::pack4_sat_s8(q[8], q[9], q[10], q[11]);
+    out.w = (int)ptx::pack4_sat_s8(q[12], q[13], q[14], q[15]);
+    *reinterpret_cast<int4*>(y + ((size_t)bc * row + (size_t)t16 * 16)) = out;
 }
 
 }  // namespace qasr

@@ -204,6 +204,13 @@ __device__ __forceinline__ int mad_hi64(int a, int b, long long c) {
         : "=r"(lo), "=r"(hi) : "r"(a), "r"(b), "r"((int)c), "r"((int)(c >> 32)));
     return hi;
 }
+// Byte B of a word, sign-extended: one prmt whose selector replicates the byte's sign over the upper three bytes.
+template <int B>
+__device__ __forceinline__ int sext_byte(uint32_t w) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, 0, %2;" : "=r"(d) : "r"(w), "n"(B | ((8 | B) << 4) | ((8 | B) << 8) | ((8 | B) << 12)));
+    return (int)d;
+}
 // max(byte, 0) on four packed int8: the sign of every byte replicated over the byte, then cleared.
 __device__ __forceinline__ uint32_t relu4_s8(uint32_t w) {
     uint32_t sign;

@@ -72,13 +72,6 @@ struct ResidualOne {
     int m0, s0, h0;    // the layer's own output: multiplier, shift, 2^(shift-1)
     int m1, s1, h1;    // the residual tensor
 };
-// Byte B of a word, sign-extended: one prmt whose selector replicates the byte's sign over the upper three bytes.
-template <int B>
-__device__ __forceinline__ int sext_byte(uint32_t w) {
-    uint32_t d;
-    asm("prmt.b32 %0, %1, 0, %2;" : "=r"(d) : "r"(w), "n"(B | ((8 | B) << 4) | ((8 | B) << 8) | ((8 | B) << 12)));
-    return (int)d;
-}
 template <bool RELU, bool S32>      // S32: every lane's shift is exactly 32, the high word is the requantised value
 __device__ __forceinline__ int4 epilogue16_res1(const uint32_t (&r)[16], const ChannelRq& rq, const int4& res,
                                                 const ResidualOne& t) {
@@ -90,7 +83,7 @@ __device__ __forceinline__ int4 epilogue16_res1(const uint32_t (&r)[16], const C
         const int hi = ptx::mad_hi64((int)r[i], rq.m, rq.c64);
         const int a = clamp_i8(S32 ? hi : hi >> sh);
         const uint32_t w = words[i >> 2];
-        const int rb = (i & 3) == 0 ? sext_byte<0>(w) : (i & 3) == 1 ? sext_byte<1>(w) : (i & 3) == 2 ? sext_byte<2>(w) : sext_byte<3>(w);
+        const int rb = (i & 3) == 0 ? ptx::sext_byte<0>(w) : (i & 3) == 1 ? ptx::sext_byte<1>(w) : (i & 3) == 2 ? ptx::sext_byte<2>(w) : ptx::sext_byte<3>(w);
         q[i] = ((a * t.m0 + t.h0) >> t.s0) + ((rb * t.m1 + t.h1) >> t.s1);
     }
     uint4 o;
