@@ -421,6 +421,17 @@ def run_ours(args):
             step()
         ablation = {"side_branch_off_ms_per_step": off_ms / min(args.steps, 30),
                     "note": "residual projections launched in table order on the main chain (QASR_OPT_SIDE_BRANCH = 0)"}
+        if any(L["kind"] == "dense" for L in model["layers"]):
+            # K-tap layers: the same step with a transpose kernel in front of every such layer instead of the
+            # frame-major second output of the layer before it
+            ctx.set_option(q.OPT_FRAME_MAJOR_OUTPUT, 0)
+            for _ in range(3):
+                step()
+            tr_ms, _ = timed(step, min(args.steps, 30))
+            ctx.set_option(q.OPT_FRAME_MAJOR_OUTPUT, 1)
+            for _ in range(3):
+                step()
+            ablation["frame_major_output_off_ms_per_step"] = tr_ms / min(args.steps, 30)
         ctx.poll_status()
 
     # per-kernel durations: the same step launched kernel by kernel between CUDA events

@@ -110,6 +110,11 @@ int qasr_poll_status(qasr_ctx* ctx);
  * main chain's kernels leave idle, and is joined in front of the first layer that needs it.  Results do not depend
  * on the option. */
 #define QASR_OPT_SIDE_BRANCH 8
+/* QASR_OPT_FRAME_MAJOR_OUTPUT (default 1): inside qasr_encoder_forward a K-tap convolution on the tensor cores
+ * whose output the next K-tap convolution of the table reads (stride 1) writes that output a second time from
+ * its epilogue, frame-major, into the workspace, so that the reader needs no transpose kernel in front of it
+ * (Sec. 3's Jasper blocks are runs of such layers).  Results do not depend on the option. */
+#define QASR_OPT_FRAME_MAJOR_OUTPUT 9
 int qasr_set_option(qasr_ctx* ctx, int option, int value);
 
 /* One kernel launch seen in profile mode: which table layer it belongs to (-1 outside

@@ -6,7 +6,7 @@ Importing it without the built library raises ImportError -- there is no CPU fal
 """
 from .binding import (NOALLOC_SCRATCH_BYTES, tcs_block_noalloc, Context, DeviceModel, QasrError, QasrLayer, QasrRequant, lib, lib_path,
                       OPT_GRAPH, OPT_TENSOR_CORES, OPT_PROFILE, OPT_STATIC_WEIGHTS, OPT_GEMM_FRAME_TILE,
-                      OPT_DW_FRAME_TILE, OPT_SIDE_BRANCH, MAX_TERMS)
+                      OPT_DW_FRAME_TILE, OPT_SIDE_BRANCH, OPT_FRAME_MAJOR_OUTPUT, MAX_TERMS)
 
 __all__ = ["NOALLOC_SCRATCH_BYTES", "tcs_block_noalloc", "Context", "DeviceModel", "QasrError", "QasrLayer", "QasrRequant", "lib", "lib_path",
-           "OPT_GRAPH", "OPT_TENSOR_CORES", "OPT_PROFILE", "OPT_STATIC_WEIGHTS", "OPT_GEMM_FRAME_TILE", "OPT_DW_FRAME_TILE", "OPT_SIDE_BRANCH", "MAX_TERMS"]
+           "OPT_GRAPH", "OPT_TENSOR_CORES", "OPT_PROFILE", "OPT_STATIC_WEIGHTS", "OPT_GEMM_FRAME_TILE", "OPT_DW_FRAME_TILE", "OPT_SIDE_BRANCH", "OPT_FRAME_MAJOR_OUTPUT", "MAX_TERMS"]

@@ -12,7 +12,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 MAX_TERMS = 12
 OPT_GRAPH, OPT_TENSOR_CORES, OPT_PROFILE, OPT_STATIC_WEIGHTS = 1, 2, 4, 5
-OPT_GEMM_FRAME_TILE, OPT_DW_FRAME_TILE, OPT_SIDE_BRANCH = 6, 7, 8
+OPT_GEMM_FRAME_TILE, OPT_DW_FRAME_TILE, OPT_SIDE_BRANCH, OPT_FRAME_MAJOR_OUTPUT = 6, 7, 8, 9
 LAYER_KINDS = {"dw": 1, "pw": 2, "dense": 3, "tcs": 4, "add": 5, "glu": 6}
 
 

@@ -53,6 +53,8 @@ struct ConvParams {
     uint16_t tap_row[128];         // stage row at which tap k of the tile's first output frame starts
     int BN, tiles_t, m_tiles, m_groups, n_items, c_chunks;
     int x_stages, w_stages, x_stage_bytes, out_bytes;
+    int dual;                      // the output is also written frame-major [B][T][C_out] (tmYt); its staging
+                                   // tiles, one [BN frames][32 channels] per quarter, follow the channel-major ones
     const int32_t* bias;
     const int32_t* mult;
     const uint8_t* shift;
@@ -85,7 +87,8 @@ __device__ __forceinline__ void conv_item_coords(const ConvParams& p, int item, 
 
 __global__ void __launch_bounds__(CV_THREADS, 1)
 conv_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-                  const __grid_constant__ CUtensorMap tmY, const ConvParams p) {
+                  const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmYt,
+                  const ConvParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const int XS = p.x_stages, WS = p.w_stages;
@@ -127,6 +130,7 @@ conv_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         ptx::tma_prefetch_desc(&tmW);
         ptx::tma_prefetch_desc(&tmX);
         ptx::tma_prefetch_desc(&tmY);
+        if (p.dual) ptx::tma_prefetch_desc(&tmYt);
     }
     // everything above overlaps the tail of the previous kernel; its results are needed from here on
     ptx::grid_dep_launch();
@@ -243,6 +247,7 @@ conv_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         const int c_hi = (part + 1) * n_chunks / CV_EPI_PARTS;
         const bool issuer = part == 0 && lane == 0;   // issues this quarter's TMA stores
         uint8_t* Oq = Os + quarter * 32 * p.BN;       // [32 channels][BN] dense staging sub-tile
+        uint8_t* Otq = Os + (CV_BM + quarter * 32) * p.BN;   // [BN frames][32 channels], the frame-major twin
         uint32_t acount = 0, qcount = 0;
         bool ok = true;
         auto quarter_sync = [&]() -> bool {
@@ -315,6 +320,14 @@ conv_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                         out = epilogue16(p, e, r, t, e.valid_o && t < p.T);
                     }
                     *reinterpret_cast<int4*>(orow + c * 16) = out;
+                    if (p.dual) {
+                        // the same 16 frames of this lane's channel, one byte per frame row: the 32 lanes of a
+                        // warp fill 32 consecutive bytes of a row per store (one wavefront)
+                        uint8_t* const ot = Otq + c * 16 * 32 + lane;
+                        const uint32_t wd[4] = {(uint32_t)out.x, (uint32_t)out.y, (uint32_t)out.z, (uint32_t)out.w};
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) ot[i * 32] = (uint8_t)(wd[i >> 2] >> (8 * (i & 3)));
+                    }
                 }
                 // accumulator drained: hand the TMEM buffer back to the MMA warp
                 ptx::tc_fence_before();
@@ -329,6 +342,11 @@ conv_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                             "cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
                             ::"l"(&tmY), "r"(t0), "r"(m * CV_BM + quarter * 32), "r"(b), "r"(ptx::smem_u32(Oq))
                             : "memory");
+                        if (p.dual)     // box: 32 channels x BN frames; frames >= T and channels >= C_out are clipped
+                            asm volatile(
+                                "cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
+                                ::"l"(&tmYt), "r"(m * CV_BM + quarter * 32), "r"(t0), "r"(b), "r"(ptx::smem_u32(Otq))
+                                : "memory");
                         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                     }
                 }
@@ -466,6 +484,8 @@ int qasr_launch_conv_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
     const size_t xt_bytes = up256((size_t)a.B * P * Tp * a.C_in);
     const size_t wt_bytes = up256((size_t)a.K * a.C_out * a.C_in);
     if (a.scratch_bytes < xt_bytes + (a.wt ? 0 : wt_bytes)) return 0;
+    // the frame-major second output: int8 results, whole 16-byte rows
+    const bool dual = a.yt && a.y && a.C_out % 16 == 0 && ((uintptr_t)a.yt & 15u) == 0;
 
     ConvParams p;
     memset(&p, 0, sizeof(p));
@@ -510,7 +530,8 @@ int qasr_launch_conv_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
         p.tap_row[k] = (uint16_t)(plane * p.R + (row - p.row_base));
     }
     p.x_stage_bytes = P * p.R * 128;
-    p.out_bytes = a.y ? (CV_BM * p.BN + 1023) / 1024 * 1024 : 0;
+    p.dual = dual ? 1 : 0;
+    p.out_bytes = a.y ? ((dual ? 2 : 1) * CV_BM * p.BN + 1023) / 1024 * 1024 : 0;
     const size_t fixed = 1024 + p.out_bytes + sizeof(ConvSharedTail);
     p.x_stages = 3;
     long long room = (long long)kConvSmemLimit - (long long)fixed - (long long)p.x_stages * p.x_stage_bytes;
@@ -524,7 +545,7 @@ int qasr_launch_conv_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
 
     int8_t* xt = (int8_t*)a.scratch;
     int8_t* wt = a.wt ? (int8_t*)a.wt : xt + xt_bytes;
-    CUtensorMap tmW, tmX, tmY;
+    CUtensorMap tmW, tmX, tmY, tmYt;
     {
         cuuint64_t dims[3] = {(cuuint64_t)a.C_in, (cuuint64_t)a.C_out, (cuuint64_t)a.K};
         cuuint64_t strides[2] = {(cuuint64_t)a.C_in, (cuuint64_t)a.C_in * a.C_out};
@@ -545,8 +566,15 @@ int qasr_launch_conv_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
     } else {
         tmY = tmX;   // unused by the int32-output path
     }
+    tmYt = tmY;      // unused without the second output
+    if (dual) {
+        cuuint64_t dims[3] = {(cuuint64_t)a.C_out, (cuuint64_t)a.T_out, (cuuint64_t)a.B};
+        cuuint64_t strides[2] = {(cuuint64_t)a.C_out, (cuuint64_t)a.C_out * a.T_out};
+        cuuint32_t box[3] = {32u, (cuuint32_t)p.BN, 1u};
+        if (!qasr_encode_map_u8(ctx, &tmYt, a.yt, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE)) return QASR_ERR_CUDA;
+    }
 
-    {
+    if (!a.xt_ready) {
         QasrLaunchScope ls(ctx, QASR_K_CONV_PREP, 0, 2.0 * a.B * a.C_in * a.T);
         dim3 grid((a.T + TR_F - 1) / TR_F, (a.C_in + TR_C - 1) / TR_C, a.B);
         transpose_frames_kernel<<<grid, 256, 0, ctx->stream>>>(a.x, xt, a.C_in, a.T, P, Tp);
@@ -569,10 +597,13 @@ int qasr_launch_conv_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
     const size_t smem = fixed + (size_t)p.x_stages * p.x_stage_bytes + (size_t)p.w_stages * CV_W_STAGE_BYTES;
     const int grid = p.n_items < qasr_grid_slots(ctx) ? p.n_items : qasr_grid_slots(ctx);
     QasrLaunchScope ls(ctx, QASR_K_CONV_TC, qasr_conv_macs(a), qasr_conv_bytes(a));
-    cudaError_t e = qasr_launch_overlapped(ctx, conv_i8_tc_kernel, dim3(grid), dim3(CV_THREADS), smem, tmW, tmX, tmY, p);
+    ctx->hold_early_launch = ctx->grid_cap > 0;      // a side branch shares the GPU
+    cudaError_t e = qasr_launch_overlapped(ctx, conv_i8_tc_kernel, dim3(grid), dim3(CV_THREADS), smem, tmW, tmX, tmY, tmYt, p);
+    ctx->hold_early_launch = false;
     if (e != cudaSuccess) {
         snprintf(ctx->err, sizeof(ctx->err), "conv_i8_tc_kernel launch failed: %s", cudaGetErrorString(e));
         return QASR_ERR_CUDA;
     }
+    ctx->yt_written = dual;
     return 1;
 }

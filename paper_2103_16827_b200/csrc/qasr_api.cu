@@ -128,6 +128,7 @@ extern "C" int qasr_set_option(qasr_ctx* ctx, int option, int value) {
         case QASR_OPT_TENSOR_CORES: ctx->opt_tc = value != 0; break;
         case QASR_OPT_PROFILE: ctx->profiling = value != 0; break;
         case QASR_OPT_SIDE_BRANCH: ctx->opt_side = value != 0; break;
+        case QASR_OPT_FRAME_MAJOR_OUTPUT: ctx->opt_dual_out = value != 0; break;
         case QASR_OPT_GEMM_FRAME_TILE:
         case QASR_OPT_DW_FRAME_TILE:
             if (value != 0 && (value < 16 || value > 256 || value % 16 != 0))
@@ -477,6 +478,9 @@ struct TablePlan {
     std::vector<BufState> bufs;   // index = buffer id; 0 = encoder input
     std::vector<int> t_in, t_out; // per layer
     size_t scratch_offset = 0, scratch_bytes = 0;
+    // second home of a frame-major input copy: a K-tap convolution reads its own copy from one region while its
+    // epilogue writes the next K-tap convolution's copy into the other
+    size_t scratch2_offset = 0, scratch2_bytes = 0;
     std::vector<size_t> wt_offset;   // per layer: home of its regrouped weights (implicit-GEMM path), or SIZE_MAX
     size_t total = 0;
     int C_last = 0, T_last = 0;
@@ -580,6 +584,7 @@ int plan_table(const qasr_layer* tb, int n, int B, int C_in, int T, TablePlan& p
                 // weights get a place of their own so that they can outlive the call
                 const size_t sb = qasr_conv_tc_input_bytes(B, L.C_in, T_i, L.stride);
                 if (sb > p.scratch_bytes) p.scratch_bytes = sb;
+                if (L.stride == 1 && sb > p.scratch2_bytes) p.scratch2_bytes = sb;
                 p.wt_offset[li] = wt_total;
                 wt_total += qasr_conv_tc_weight_bytes(L.C_in, L.C_out, L.K);
             }
@@ -606,6 +611,8 @@ int plan_table(const qasr_layer* tb, int n, int B, int C_in, int T, TablePlan& p
     }
     p.scratch_offset = off;
     off += (p.scratch_bytes + 255) / 256 * 256;
+    p.scratch2_offset = off;
+    off += (p.scratch2_bytes + 255) / 256 * 256;
     for (int li = 0; li < n; ++li)
         if (p.wt_offset[li] != SIZE_MAX) p.wt_offset[li] += off;
     off += wt_total;
@@ -681,6 +688,18 @@ static int enqueue_table(qasr_ctx* ctx, const qasr_layer* tb, int n, const Table
         bool reads(int b) const { for (int v : in_bufs) if (v == b) return true; return false; }
         bool writes(int b) const { for (int v : out_bufs) if (v == b) return true; return false; }
     } side;
+    // Frame-major copy of a tensor that a K-tap convolution's epilogue has already left in one of the two scratch
+    // regions (buffer id, region), valid until that buffer or that region is written again.
+    int ft_buf = -1, ft_region = 0;
+    auto scratch_region = [&](int r, size_t& bytes) -> char* {
+        bytes = r ? p.scratch2_bytes : p.scratch_bytes;
+        return ws + (r ? p.scratch2_offset : p.scratch_offset);
+    };
+    // A layer that takes the scratch-using convolution path (anything the pointwise GEMM does not take).
+    auto wants_scratch = [&](const qasr_layer& Q, int T_out) {
+        return (Q.kind == QASR_LAYER_DENSE || Q.kind == QASR_LAYER_PW) &&
+               !qasr_conv_shape_fits_gemm(Q.C_in, Q.K, Q.stride, Q.dilation, T_out);
+    };
     const int main_slots = 128;
     const bool side_ok = capturing && ctx->opt_side && ctx->opt_tc && ctx->encode_tiled && !ctx->profiling &&
                          ctx->sm_count >= main_slots + 16;
@@ -718,6 +737,7 @@ static int enqueue_table(qasr_ctx* ctx, const qasr_layer* tb, int n, const Table
                 if (side.writes(L.term_buf[j])) hazard = true;
             if (hazard && (rc = join_side())) return rc;
         }
+        if (!L.out_int32 && L.out_buf == ft_buf) ft_buf = -1;     // the tensor is overwritten: its copy is stale
         if (L.kind == QASR_LAYER_ADD) {
             QasrTerms t;
             memset(&t, 0, sizeof(t));
@@ -792,15 +812,48 @@ static int enqueue_table(qasr_ctx* ctx, const qasr_layer* tb, int n, const Table
             } else if (L.kind == QASR_LAYER_TCS) {
                 QasrDwArgs d{in, L.w_dw, L.rq_dw.mult, L.rq_dw.shift, nullptr, B, L.C_in, T_i, T_o, L.K, L.stride, L.dilation};
                 a.T = T_o; a.T_out = T_o; a.K = 1; a.stride = 1; a.dilation = 1;
+                if (ft_region == 0) ft_buf = -1;        // the depthwise output goes to the first scratch region
                 rc = run_tcs(ctx, d, a, ws + p.scratch_offset);
             } else {
                 a.T = T_i; a.T_out = T_o; a.K = L.K; a.stride = L.stride; a.dilation = L.dilation;
-                a.scratch = ws + p.scratch_offset; a.scratch_bytes = p.scratch_bytes;
+                // the frame-major input copy: where the producing layer left it, else region 0 (transposed there)
+                int in_region = 0;
+                if (wants_scratch(L, T_o)) {
+                    if (ft_buf == L.in_buf && L.stride == 1) {
+                        in_region = ft_region;
+                        a.xt_ready = 1;
+                    } else if (ft_region == 0) {
+                        ft_buf = -1;
+                    }
+                }
+                a.scratch = scratch_region(in_region, a.scratch_bytes);
                 if (p.wt_offset[li] != SIZE_MAX) {
                     a.wt = ws + p.wt_offset[li];
                     a.wt_ready = weights_ready ? 1 : 0;
                 }
+                // Second, frame-major output for the K-tap convolution that reads this tensor next: the first
+                // scratch-using layer that follows (pointwise layers on the GEMM path in between use none),
+                // reached before anything overwrites the tensor. It goes to the region this layer does not read.
+                if (ctx->opt_dual_out && !L.out_int32 && wants_scratch(L, T_o)) {
+                    for (int lj = li + 1; lj < n; ++lj) {
+                        const qasr_layer& N = tb[lj];
+                        const bool gemm_pw = N.kind == QASR_LAYER_PW && !wants_scratch(N, p.t_out[lj]);
+                        if (gemm_pw && N.out_buf != L.out_buf) continue;
+                        size_t rbytes = 0;
+                        char* const home = scratch_region(1 - in_region, rbytes);
+                        if (wants_scratch(N, p.t_out[lj]) && N.in_buf == L.out_buf && N.stride == 1 &&
+                            N.out_buf != L.out_buf && (size_t)B * L.C_out * T_o <= rbytes)
+                            a.yt = (int8_t*)home;
+                        break;
+                    }
+                }
+                ctx->yt_written = false;
                 rc = run_conv(ctx, a);
+                if (a.yt) {
+                    // whatever the other region held is gone, whether or not the tensor-core kernel ran
+                    ft_buf = ctx->yt_written ? L.out_buf : -1;
+                    ft_region = 1 - in_region;
+                }
             }
         }
         if (rc) return rc;

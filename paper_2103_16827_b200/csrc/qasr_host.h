@@ -46,6 +46,14 @@ struct qasr_ctx {
     // Side branch of a captured layer table: a convolution whose result is needed only several layers later
     // (a block's residual projection) runs on a second stream, on the SMs the main chain leaves idle.
     bool opt_side = true;
+    // A K-tap convolution on the tensor cores writes its output a second time, frame-major, where the next
+    // K-tap convolution of the table reads it (that one then needs no transpose kernel).
+    bool opt_dual_out = true;
+    // Set around a launch whose CTAs must not become resident before the previous kernel has ended: while a side
+    // branch is pending, early CTAs of a long main-chain kernel would sit in their dependency wait on the very SMs
+    // the branch's next kernel needs.
+    bool hold_early_launch = false;
+    bool yt_written = false;                     // set by the launch that wrote QasrConvArgs::yt
     int grid_cap = 0;                            // > 0: persistent kernels launch at most this many CTAs
     cudaStream_t side_stream = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_side = nullptr;
@@ -152,7 +160,7 @@ inline cudaError_t qasr_launch_overlapped(qasr_ctx* ctx, void (*kernel)(KArgs...
     cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = ctx->stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = ctx->opt_pdl ? 1 : 0;
+    attr[0].val.programmaticStreamSerializationAllowed = ctx->opt_pdl && !ctx->hold_early_launch ? 1 : 0;
     cfg.attrs = attr; cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }

@@ -42,6 +42,9 @@ struct QasrConvArgs {
     size_t scratch_bytes;
     void* wt;                 // optional separate home of the regrouped weights (else they follow the input copy in scratch)
     int wt_ready;             // wt already holds this layer's regrouped weights: skip the regrouping kernel
+    int8_t* yt;               // optional second home of the output, frame-major [B][T_out][C_out]: what a K-tap
+                              // convolution that reads this tensor next (stride 1) wants as its input copy
+    int xt_ready;             // scratch already holds this layer's frame-major input copy: skip the transpose
 };
 
 struct QasrDwArgs {
