@@ -42,7 +42,11 @@ constexpr int CV_EPI_WARPS = 4 * CV_EPI_PARTS;
 constexpr int CV_THREADS = 64 + 32 * CV_EPI_WARPS;
 constexpr int CV_ACC_STRIDE = 256;
 constexpr int CV_TMEM_COLS = 512;
-constexpr int CV_W_STAGE_BYTES = CV_BM * CV_BK;
+constexpr int CV_W_BLOCK_BYTES = CV_BM * CV_BK;          // one tap's [128 x 128] weight block
+// A weight stage holds the blocks of several consecutive taps (ConvParams::w_taps; one TMA box, one barrier
+// round trip and one commit per 4 * w_taps MMAs): the issuing warp's fixed cost per round is what this kernel's
+// rate depends on.
+constexpr int CV_MAX_W_TAPS = 4;
 
 struct ConvParams {
     int B, C_in, C_out, T;         // T = output frames per utterance
@@ -53,6 +57,7 @@ struct ConvParams {
     uint16_t tap_row[128];         // stage row at which tap k of the tile's first output frame starts
     int BN, tiles_t, m_tiles, m_groups, n_items, c_chunks;
     int x_stages, w_stages, x_stage_bytes, out_bytes;
+    int w_taps;                    // taps per weight stage
     int dual;                      // the output is also written frame-major [B][T][C_out] (tmYt); its staging
                                    // tiles, one [BN frames][32 channels] per quarter, follow the channel-major ones
     const int32_t* bias;
@@ -94,7 +99,9 @@ conv_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     const int XS = p.x_stages, WS = p.w_stages;
     uint8_t* Xs = smem;                                          // XS stages of P * R rows of 128 bytes
     uint8_t* Ws = Xs + (size_t)XS * p.x_stage_bytes;             // WS stages of 16 KiB
-    uint8_t* Os = Ws + (size_t)WS * CV_W_STAGE_BYTES;            // [128 channels][BN frames] output staging
+    const int W_TAPS = p.w_taps;
+    const uint32_t W_STAGE_BYTES = (uint32_t)W_TAPS * CV_W_BLOCK_BYTES;
+    uint8_t* Os = Ws + (size_t)WS * W_STAGE_BYTES;            // [128 channels][BN frames] output staging
     ConvSharedTail* sh = (ConvSharedTail*)(Os + p.out_bytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -165,12 +172,12 @@ conv_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                             ptx::tma_load_3d(xs_base + xs * x_stage_bytes + pl * plane_bytes, &tmX,
                                              cc * CV_BK, t0 + row_base, b * P + pl, xbar);
                         if (++xs == XS) { xs = 0; xph ^= 1u; }
-                        for (int k = 0; k < K; ++k) {
+                        for (int k = 0; k < K; k += W_TAPS) {     // taps >= K of the last box arrive as zeros, never used
                             ok = ptx::mbar_try(wempty0 + ws * 8, wph) || ptx::mbar_wait(wempty0 + ws * 8, wph, abort_flag, p.status);
                             if (!ok) break;
                             const uint32_t wbar = wfull0 + ws * 8;
-                            ptx::mbar_expect_tx(wbar, CV_W_STAGE_BYTES);
-                            ptx::tma_load_3d(ws_base + ws * CV_W_STAGE_BYTES, &tmW, cc * CV_BK, m * CV_BM, k, wbar);
+                            ptx::mbar_expect_tx(wbar, W_STAGE_BYTES);
+                            ptx::tma_load_3d(ws_base + ws * W_STAGE_BYTES, &tmW, cc * CV_BK, m * CV_BM, k, wbar);
                             if (++ws == WS) { ws = 0; wph ^= 1u; }
                         }
                     }
@@ -213,18 +220,21 @@ conv_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                         if (!ok) break;
                         const uint64_t b_stage = b_desc0 + (uint32_t)xs * x_stage16;
                         const int ksteps = cc == c_chunks - 1 ? ksteps_last : CV_BK / 32;
-                        for (int k = 0; k < K; ++k) {
+                        for (int k = 0; k < K; k += W_TAPS) {
                             ok = ptx::mbar_try(wfull0 + ws * 8, wph) || ptx::mbar_wait(wfull0 + ws * 8, wph, abort_flag, p.status);
                             ok = __all_sync(0xffffffffu, ok);
                             if (!ok) break;
                             ptx::tc_fence_after();
-                            const uint64_t ad = a_desc0 + (uint32_t)ws * (CV_W_STAGE_BYTES >> 4);
-                            const uint64_t bd = b_stage + (uint32_t)p.tap_row[k] * 8u;      // whole 128-byte rows
+                            uint64_t ad = a_desc0 + (uint32_t)ws * (W_STAGE_BYTES >> 4);
+                            const int taps_here = min(W_TAPS, K - k);
                             if (ptx::elect_one()) {
+                                for (int u = 0; u < taps_here; ++u, ad += CV_W_BLOCK_BYTES >> 4) {
+                                    const uint64_t bd = b_stage + (uint32_t)p.tap_row[k + u] * 8u;      // whole 128-byte rows
 #pragma unroll
-                                for (int j = 0; j < CV_BK / 32; ++j) {
-                                    if (j < ksteps)
-                                        ptx::mma_i8(d_tmem, ad + 2 * j, bd + 2 * j, idesc, j == 0 ? accumulate : 1u);   // 32 channels further
+                                    for (int j = 0; j < CV_BK / 32; ++j) {
+                                        if (j < ksteps)
+                                            ptx::mma_i8(d_tmem, ad + 2 * j, bd + 2 * j, idesc, (u | j) == 0 ? accumulate : 1u);   // 32 channels further
+                                    }
                                 }
                                 ptx::tc_commit(wempty0 + ws * 8);
                             }
@@ -535,12 +545,17 @@ int qasr_launch_conv_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
     const size_t fixed = 1024 + p.out_bytes + sizeof(ConvSharedTail);
     p.x_stages = 3;
     long long room = (long long)kConvSmemLimit - (long long)fixed - (long long)p.x_stages * p.x_stage_bytes;
-    if (room < 5LL * CV_W_STAGE_BYTES) {
+    if (room < 6LL * CV_W_BLOCK_BYTES) {
         p.x_stages = 2;
         room = (long long)kConvSmemLimit - (long long)fixed - (long long)p.x_stages * p.x_stage_bytes;
     }
-    if (room < 3LL * CV_W_STAGE_BYTES) return 0;
-    p.w_stages = (int)(room / CV_W_STAGE_BYTES);
+    if (room < 3LL * CV_W_BLOCK_BYTES) return 0;
+    // taps per weight stage: two where that leaves a ring of at least three stages (measured on 768 -> 768, K = 13,
+    // B = 64: 2306 TOP/s with one tap per stage, 2709 with two, 2725 / 2703 with three / four)
+    const int blocks = (int)(room / CV_W_BLOCK_BYTES);
+    p.w_taps = blocks >= 6 ? 2 : 1;
+    if (p.w_taps > a.K) p.w_taps = a.K;
+    p.w_stages = blocks / p.w_taps;
     if (p.w_stages > CV_MAX_WS) p.w_stages = CV_MAX_WS;
 
     int8_t* xt = (int8_t*)a.scratch;
@@ -549,7 +564,7 @@ int qasr_launch_conv_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
     {
         cuuint64_t dims[3] = {(cuuint64_t)a.C_in, (cuuint64_t)a.C_out, (cuuint64_t)a.K};
         cuuint64_t strides[2] = {(cuuint64_t)a.C_in, (cuuint64_t)a.C_in * a.C_out};
-        cuuint32_t box[3] = {(cuuint32_t)CV_BK, (cuuint32_t)CV_BM, 1u};
+        cuuint32_t box[3] = {(cuuint32_t)CV_BK, (cuuint32_t)CV_BM, (cuuint32_t)p.w_taps};
         if (!qasr_encode_map_u8(ctx, &tmW, wt, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) return QASR_ERR_CUDA;
     }
     {
@@ -594,7 +609,7 @@ int qasr_launch_conv_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
             return QASR_ERR_CUDA;
         }
     }
-    const size_t smem = fixed + (size_t)p.x_stages * p.x_stage_bytes + (size_t)p.w_stages * CV_W_STAGE_BYTES;
+    const size_t smem = fixed + (size_t)p.x_stages * p.x_stage_bytes + (size_t)p.w_stages * p.w_taps * CV_W_BLOCK_BYTES;
     const int grid = p.n_items < qasr_grid_slots(ctx) ? p.n_items : qasr_grid_slots(ctx);
     QasrLaunchScope ls(ctx, QASR_K_CONV_TC, qasr_conv_macs(a), qasr_conv_bytes(a));
     ctx->hold_early_launch = ctx->grid_cap > 0;      // a side branch shares the GPU
