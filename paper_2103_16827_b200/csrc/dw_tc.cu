@@ -71,6 +71,10 @@ struct Params {
     int nsb, NS, NS_last;            // nsb - 1 sub-blocks of NS columns, the last of NS_last
     int Kspan;                       // K extent of one sub-block's MMA chain (multiple of 32)
     int a_kblocks;                   // 128-byte K blocks of A
+    int a_kblocks_ld, last_w;        // K blocks that are loaded, and the bytes of the last of them (multiple of 16):
+                                     // behind the last byte any output needs the band is zero, so whatever the
+                                     // stage still holds there multiplies zeros (integers: no NaN can arise)
+    int ksteps_last;                 // 32-byte K steps of the last (narrower) sub-block's MMA chain
     int b_rows;                      // rows of the band matrix = widest sub-block
     int band_chunks;                 // 16-byte chunks a band row can touch
     int a_bytes, b_bytes;            // per stage
@@ -119,8 +123,8 @@ __device__ __forceinline__ int4 requant16_dw(const uint32_t (&r)[16], int mn, lo
 }
 
 __global__ void __launch_bounds__(THREADS, 1)
-dw_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY,
-             const __grid_constant__ CUtensorMap tmYw, const Params p) {
+dw_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmXl,
+             const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmYw, const Params p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* const A0 = smem;
@@ -182,7 +186,7 @@ dw_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
         it.c = item / p.MT;
         mtile_coords(p, item - it.c * p.MT, it.tile0, it.b0);
         it.n_tiles = min(p.tpm, p.tiles - it.tile0);
-        it.n_boxes = it.n_tiles * p.a_kblocks;
+        it.n_boxes = it.n_tiles * p.a_kblocks_ld;
         it.kb = bbox / it.n_tiles;                 // the box this thread issues (if bbox < n_boxes)
         it.ti = bbox - it.kb * it.n_tiles;
         return it;
@@ -190,6 +194,7 @@ dw_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
     ItemAt at = locate(bgrp);
     if (threadIdx.x == 0) {   // kernel parameters: fetch them while the previous kernel drains
         ptx::tma_prefetch_desc(&tmX);
+        ptx::tma_prefetch_desc(&tmXl);
         ptx::tma_prefetch_desc(&tmY);
         ptx::tma_prefetch_desc(&tmYw);
     }
@@ -219,7 +224,8 @@ dw_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
             // frames outside [0, T) are filled with zeros by the copy engine
             auto load_windows = [&]() {
                 if (bbox < n_boxes)
-                    ptx::tma_load_3d(ptx::smem_u32(Astage + at.kb * A_KBLOCK_BYTES + at.ti * p.rows_b * 128), &tmX,
+                    ptx::tma_load_3d(ptx::smem_u32(Astage + at.kb * A_KBLOCK_BYTES + at.ti * p.rows_b * 128),
+                                     at.kb == p.a_kblocks_ld - 1 ? &tmXl : &tmX,
                                      (tile0 + at.ti) * p.NT * p.stride - p.padL + 128 * at.kb, c, b0, ptx::smem_u32(&sh->full[grp]));
             };
             const bool first_use = n == (uint32_t)grp;     // the stage has never been used: nothing to wait for
@@ -246,7 +252,8 @@ dw_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
             if (tid == 0) {
                 const bool ok = first_use || ptx::mbar_wait(ptx::smem_u32(&sh->empty[grp]), ((n >> 1) & 1u) ^ 1u, abort_flag, p.status);
                 sh->build_ok[grp] = ok ? 1 : 0;
-                if (ok) ptx::mbar_expect_tx(ptx::smem_u32(&sh->full[grp]), (uint32_t)(n_boxes * p.rows_b * 128));
+                if (ok) ptx::mbar_expect_tx(ptx::smem_u32(&sh->full[grp]),
+                                            (uint32_t)(at.n_tiles * p.rows_b * (128 * (p.a_kblocks_ld - 1) + p.last_w)));
             }
             asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "n"(BUILD_GROUP_THREADS) : "memory");   // tap line complete, go/no-go known
             if (!sh->build_ok[grp]) break;
@@ -313,12 +320,13 @@ dw_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
                 if (ptx::elect_one()) {
                 for (int sb = 0; sb < nsb; ++sb) {
                     const uint32_t idesc = sb == nsb - 1 ? idesc_last : idesc_mid;
+                    const int ks = sb == nsb - 1 ? p.ksteps_last : ksteps;
                     uint32_t within = (uint32_t)koff & 127u;
                     uint64_t ad = a_stage + (((uint32_t)koff >> 7) << 10) + (within >> 4);
                     uint64_t bd = b_stage;
                     uint32_t b_within = 0;
                     uint32_t accumulate = 0;
-                    for (int j = 0; j < ksteps; ++j) {
+                    for (int j = 0; j < ks; ++j) {
                         ptx::mma_i8(d_tmem + sb * NS, ad, bd, idesc, accumulate);
                         accumulate = 1;
                         ad += 2;
@@ -373,11 +381,12 @@ dw_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
                 int tile0, b0;
                 mtile_coords(p, item - c0 * p.MT, tile0, b0);
                 const int n_tiles = min(p.tpm, p.tiles - tile0);
-                const int n_boxes = n_tiles * p.a_kblocks;
+                const int n_boxes = n_tiles * p.a_kblocks_ld;
                 uint8_t* const Astage = g ? A1 : A0;
                 for (int j = lane * EPI_WARPS + ew; j < n_boxes; j += 32 * EPI_WARPS) {
                     const int kb = j / n_tiles, ti = j - kb * n_tiles;
-                    ptx::tma_load_3d(ptx::smem_u32(Astage + kb * A_KBLOCK_BYTES + ti * p.rows_b * 128), &tmX,
+                    ptx::tma_load_3d(ptx::smem_u32(Astage + kb * A_KBLOCK_BYTES + ti * p.rows_b * 128),
+                                     kb == p.a_kblocks_ld - 1 ? &tmXl : &tmX,
                                      (tile0 + ti) * p.NT * p.stride - p.padL + 128 * kb, c0, b0, ptx::smem_u32(&sh->full[g]));
                 }
             }
@@ -550,6 +559,15 @@ int qasr_launch_dw_tc(qasr_ctx* ctx, const QasrDwArgs& a) {
         const int kga = (p.nsb - 1) * p.NS * a.stride + p.Kspan;
         p.a_kblocks = (kga + 127) / 128;
         p.band_chunks = ((a.K - 1) * a.dilation + 15) / 16 + 1;
+        {
+            // the last input byte any output of a window needs, and the K extent of the last sub-block's chain
+            const int need = (p.NT - 1) * a.stride + p.lead + (a.K - 1) * a.dilation + 1;
+            p.a_kblocks_ld = (need + 127) / 128;
+            p.last_w = ((need - 128 * (p.a_kblocks_ld - 1)) + 15) & ~15;
+            const int span_last = (p.NS_last - 1) * a.stride + p.lead + (a.K - 1) * a.dilation + 1;
+            p.ksteps_last = (span_last + 31) / 32;
+            if (p.ksteps_last > p.Kspan / 32) p.ksteps_last = p.Kspan / 32;
+        }
         p.a_bytes = p.a_kblocks * A_KBLOCK_BYTES;
         p.b_bytes = ((p.Kspan + 127) / 128) * p.b_rows * 128;     // whole 128-byte K blocks of the swizzled band
         smem = 1024 + 2 * (size_t)(p.a_bytes + p.b_bytes) + 2 * 4 * LINE_WORDS * 4 + sizeof(SharedTail) +
@@ -561,12 +579,15 @@ int qasr_launch_dw_tc(qasr_ctx* ctx, const QasrDwArgs& a) {
     p.next = ctx->prefetch;
     memset(&ctx->prefetch, 0, sizeof(ctx->prefetch));
 
-    CUtensorMap tmX;
+    CUtensorMap tmX, tmXl;
     {
         cuuint64_t dims[3] = {(cuuint64_t)a.T, (cuuint64_t)a.C, (cuuint64_t)a.B};
         cuuint64_t strides[2] = {(cuuint64_t)a.T, (cuuint64_t)a.T * a.C};
         cuuint32_t box[3] = {128u, 1u, (cuuint32_t)p.rows_b};
         if (!qasr_encode_map_u8(ctx, &tmX, a.x, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) return QASR_ERR_CUDA;
+        // the last loaded K block: only as wide as the outputs need it (same 128-byte row pitch and swizzle)
+        box[0] = (cuuint32_t)p.last_w;
+        if (!qasr_encode_map_u8(ctx, &tmXl, a.x, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) return QASR_ERR_CUDA;
     }
     CUtensorMap tmY = tmX, tmYw = tmX;     // unused without staging
     if (p.staged) {
@@ -580,7 +601,7 @@ int qasr_launch_dw_tc(qasr_ctx* ctx, const QasrDwArgs& a) {
     }
     const int grid = p.n_items < qasr_grid_slots(ctx) ? p.n_items : qasr_grid_slots(ctx);
     QasrLaunchScope ls(ctx, QASR_K_DW_TC, qasr_dw_macs(a), qasr_dw_bytes(a));
-    cudaError_t e = qasr_launch_overlapped(ctx, dw_tc_kernel, dim3(grid), dim3(THREADS), smem, tmX, tmY, tmYw, p);
+    cudaError_t e = qasr_launch_overlapped(ctx, dw_tc_kernel, dim3(grid), dim3(THREADS), smem, tmX, tmXl, tmY, tmYw, p);
     if (e != cudaSuccess) {
         snprintf(ctx->err, sizeof(ctx->err), "dw_tc_kernel launch failed: %s", cudaGetErrorString(e));
         return QASR_ERR_CUDA;
