@@ -765,6 +765,59 @@ def test_frame_major_second_output_replaces_the_transposes(q, ctx, shape):
         assert n_conv + 1 <= preps[1][0] < 2 * n_conv
 
 
+def _mixed_ktap_table(unique_bufs):
+    """K-tap layers with everything that can stand between a frame-major second output and its reader."""
+    rng = workloads.rng_for(21)
+    x = workloads.draw_input(rng, 2, 32, 256)
+    bld = workloads._Builder(rng, "live", unique_bufs, False)
+    W = workloads
+    a = bld.conv("dense", "k0", 0, 32, 64, 5, 1, 1, True, W.MS_INPUT)
+    b = bld.conv("dense", "k1", a, 64, 64, 7, 1, 1, True, W.MS_RELU)            # reads k0's frame-major copy
+    bld.release(a)
+    c = bld.tcs("t2", b, 64, 64, 9, 1, 1, True, W.MS_RELU)                      # its depthwise output takes region 0
+    bld.release(b)
+    d = bld.conv("dense", "k3", c, 64, 96, 5, 1, 1, True, W.MS_RELU)            # input from a GEMM: transposed
+    bld.release(c)
+    e = bld.conv("dense", "k4", d, 96, 96, 3, 2, 1, True, W.MS_RELU)            # stride 2: planes, transposed
+    bld.release(d)
+    f = bld.conv("dense", "k5", e, 96, 64, 5, 1, 1, True, W.MS_RELU)
+    bld.release(e)
+    g = bld.conv("pw", "p6", f, 64, 64, 1, 1, 1, False, W.MS_RELU)              # GEMM layer between k5 and its reader
+    h = bld.conv("dense", "k7", f, 64, 64, 5, 1, 2, True, W.MS_RELU, res=[g])   # reads k5's copy, adds p6
+    bld.release(f)
+    bld.release(g)
+    i = bld.conv("dense", "k8", h, 64, 48, 3, 1, 1, True, W.MS_RELU)            # 48 channels: one and a half store boxes
+    bld.release(h)
+    j = bld.conv("pw", "p9", i, 48, 80, 1, 1, 1, True, W.MS_RELU)               # pointwise off the GEMM's shapes: uses scratch
+    bld.release(i)
+    bld.conv("pw", "head", j, 80, 29, 1, 1, 1, False, W.MS_RELU, out_int32=True)
+    out_scale = (rng.uniform(0.5, 1.5, size=29) * 1e-3).astype(np.float32)
+    return {"name": "mixed_ktap", "B": 2, "T": 256, "C_in": 32, "layers": bld.layers, "out_scale": out_scale,
+            "n_bufs": bld.next_buf, "variant": "live"}, x
+
+
+@pytest.mark.parametrize("unique_bufs", [True, False])
+def test_frame_major_second_output_in_a_mixed_table(q, ctx, unique_bufs):
+    """The frame-major copies live in two scratch regions that other layers use as well (a TCS block's depthwise
+    output, transposed inputs): a table that puts a TCS block, a stride-2 layer, a pointwise GEMM and a
+    scratch-using pointwise layer between K-tap layers, with ping-pong buffers and with one buffer per layer."""
+    model, x = _mixed_ktap_table(unique_bufs)
+    wq, wf, trace = oracle.encoder_forward(model, x)
+    for on in (1, 0):
+        ctx.set_option(q.OPT_FRAME_MAJOR_OUTPUT, on)
+        try:
+            for rep in range(2):            # capture, then replay
+                gq, gf, bufs, _ = run_encoder_T(q, ctx, model, x, wq.shape[2], want_bufs=unique_bufs)
+                if unique_bufs:
+                    for L, o in zip(model["layers"][:-1], trace[:-1]):
+                        assert_same(bufs[L["out"]], o["y"], "layer %s (option %d)" % (L["name"], on))
+                assert_same(gq, wq, "logits_q (option %d, pass %d)" % (on, rep))
+                assert np.max(np.abs(gf - wf)) <= 1e-6
+        finally:
+            ctx.set_option(q.OPT_FRAME_MAJOR_OUTPUT, 1)
+    assert np.std(wq.astype(np.float64)) > 10
+
+
 def test_config3_jasper_full_batch_sampled_utterances(q, ctx):
     """JasperDR-10x5 shape at B=16, T=1600; the oracle computes utterances 0, 7 and 15 on their own."""
     model, x = workloads.config(3, variant="live")
