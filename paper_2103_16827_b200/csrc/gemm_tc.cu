@@ -50,6 +50,9 @@ struct GemmParams {
     int m_tiles, m_groups;         // 128-channel output tiles and groups they are split into
     int n_items;
     int w_stages;                  // depth of the weight ring (<= MAX_W_STAGES)
+    int w_pair;                    // a weight stage holds two K blocks: every output tile of an item but the first
+                                   // (whose blocks are wanted one by one, as the activation blocks arrive) takes one
+                                   // barrier round trip and one commit per two K blocks
     int out_bytes;                 // bytes of the output staging area (one block per epilogue warp)
     int stage_w;                   // bytes per staged row of the wider warps (16 * ceil(chunks / warps per quarter))
     const int32_t* bias;
@@ -90,9 +93,10 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                   const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    constexpr int W_STAGE_BYTES = BM * BK;
+    constexpr int W_BLOCK_BYTES = BM * BK;
     constexpr int X_BLOCK_BYTES = BK * 128;     // one (BK channels x 128 frames) swizzled block
     const int W_STAGES = p.w_stages;
+    const int W_STAGE_BYTES = p.w_pair ? 2 * W_BLOCK_BYTES : W_BLOCK_BYTES;
     const int KB = p.C_in / BK;
     uint8_t* Xs = smem;                                         // KB * NC blocks of 8 KiB
     uint8_t* Ws = Xs + (size_t)KB * p.NC * X_BLOCK_BYTES;       // W_STAGES stages of 8 KiB
@@ -156,8 +160,17 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                 ok = ptx::mbar_try(wempty0 + ws * 8, wph) || ptx::mbar_wait(wempty0 + ws * 8, wph, abort_flag, p.status);
                 if (!ok) return;
                 const uint32_t bar = wfull0 + ws * 8;
-                ptx::mbar_expect_tx(bar, W_STAGE_BYTES);
+                ptx::mbar_expect_tx(bar, W_BLOCK_BYTES);
                 ptx::tma_load_2d(ws_base + ws * W_STAGE_BYTES, &tmW, kb * BK, m * BM, bar);
+                if (++ws == W_STAGES) { ws = 0; wph ^= 1u; }
+            };
+            auto issue_w2 = [&](int m, int kb, int kb1) {       // two K blocks into one stage
+                ok = ptx::mbar_try(wempty0 + ws * 8, wph) || ptx::mbar_wait(wempty0 + ws * 8, wph, abort_flag, p.status);
+                if (!ok) return;
+                const uint32_t bar = wfull0 + ws * 8;
+                ptx::mbar_expect_tx(bar, 2 * W_BLOCK_BYTES);
+                ptx::tma_load_2d(ws_base + ws * W_STAGE_BYTES, &tmW, kb * BK, m * BM, bar);
+                ptx::tma_load_2d(ws_base + ws * W_STAGE_BYTES + W_BLOCK_BYTES, &tmW, kb1 * BK, m * BM, bar);
                 if (++ws == W_STAGES) { ws = 0; wph ^= 1u; }
             };
             // coordinates of an item; those of the first one are ready before the dependency wait returns
@@ -194,9 +207,17 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                 for (int mi = 1; mi < mc && ok; ++mi) {
                     if (++mr == mc) mr = 0;
                     kb = rot_k;
-                    for (int ki = 0; ki < KB && ok; ++ki) {
-                        issue_w(m_lo + mr, kb);
-                        if (++kb == KB) kb = 0;
+                    if (p.w_pair) {
+                        for (int ki = 0; ki < KB && ok; ki += 2) {
+                            const int kb1 = kb + 1 == KB ? 0 : kb + 1;
+                            issue_w2(m_lo + mr, kb, kb1);
+                            kb = kb1 + 1 == KB ? 0 : kb1 + 1;
+                        }
+                    } else {
+                        for (int ki = 0; ki < KB && ok; ++ki) {
+                            issue_w(m_lo + mr, kb);
+                            if (++kb == KB) kb = 0;
+                        }
                     }
                 }
                 iph ^= 1u;
@@ -236,13 +257,40 @@ gemm_i8_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                     const bool first = mi == 0, last = mi == mc - 1;
                     uint32_t accumulate = 0;
                     int kb = rot_k;
+                    if (p.w_pair && !first) {
+                        // the activation tile is resident: two K blocks per weight stage
+                        for (int ki = 0; ki < KB; ki += 2) {
+                            ok = ptx::mbar_try(wfull0 + ws * 8, wph) || ptx::mbar_wait(wfull0 + ws * 8, wph, abort_flag, p.status);
+                            ok = __all_sync(0xffffffffu, ok);
+                            if (!ok) break;
+                            ptx::tc_fence_after();
+                            const int kb1 = kb + 1 == KB ? 0 : kb + 1;
+                            const uint64_t ad = a_desc0 + (uint32_t)ws * ((uint32_t)W_STAGE_BYTES >> 4);
+                            const uint64_t bd = b_desc0 + (uint32_t)kb * x_kb16;
+                            const uint64_t bd1 = b_desc0 + (uint32_t)kb1 * x_kb16;
+                            __syncwarp();
+                            if (ptx::elect_one()) {
+#pragma unroll
+                                for (int j = 0; j < BK / 32; ++j)
+                                    ptx::mma_i8(d_tmem, ad + 2 * j, bd + 256 * j, idesc, j == 0 ? accumulate : 1u);
+#pragma unroll
+                                for (int j = 0; j < BK / 32; ++j)
+                                    ptx::mma_i8(d_tmem, ad + (W_BLOCK_BYTES >> 4) + 2 * j, bd1 + 256 * j, idesc, 1u);
+                                ptx::tc_commit(wempty0 + ws * 8);
+                                if (last) { ptx::tc_commit(xempty0 + kb * 8); ptx::tc_commit(xempty0 + kb1 * 8); }
+                            }
+                            accumulate = 1;
+                            if (++ws == W_STAGES) { ws = 0; wph ^= 1u; }
+                            kb = kb1 + 1 == KB ? 0 : kb1 + 1;
+                        }
+                    } else
                     for (int ki = 0; ki < KB; ++ki) {
                         if (first) ok = ptx::mbar_try(xfull0 + kb * 8, iph) || ptx::mbar_wait(xfull0 + kb * 8, iph, abort_flag, p.status);
                         if (ok) ok = ptx::mbar_try(wfull0 + ws * 8, wph) || ptx::mbar_wait(wfull0 + ws * 8, wph, abort_flag, p.status);
                         ok = __all_sync(0xffffffffu, ok);
                         if (!ok) break;
                         ptx::tc_fence_after();
-                        const uint64_t ad = a_desc0 + (uint32_t)ws * (W_STAGE_BYTES >> 4);
+                        const uint64_t ad = a_desc0 + (uint32_t)ws * ((uint32_t)W_STAGE_BYTES >> 4);
                         const uint64_t bd = b_desc0 + (uint32_t)kb * x_kb16;
                         __syncwarp();
                         if (ptx::elect_one()) {
@@ -516,6 +564,13 @@ int qasr_launch_gemm_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
     layout(GROUPS, p.stage_w, p.out_bytes, p.w_stages);
     const size_t fixed = 1024 + (size_t)a.C_in * p.NC * 128 + p.out_bytes + sizeof(SharedTail);
     if (p.w_stages < 2) return QASR_ERR_SHAPE;
+    // two K blocks per weight stage where an item has further output tiles after its first and the ring stays two
+    // stages deep
+    const int KB = a.C_in / BK;
+    // (512->512 at B=32 12.1 -> 11.7 us, at B=256 74.3 -> 70.5 us; the benchmark step moves by 0.25 %: its pointwise
+    // layers wait for their epilogues as much as for the MMA warp)
+    p.w_pair = KB % 2 == 0 && per_item >= 2 && p.w_stages >= 4 ? 1 : 0;
+    if (p.w_pair) p.w_stages /= 2;
     CUtensorMap tmW, tmX, tmXl, tmY, tmYw;
     {
         cuuint64_t dims[2] = {(cuuint64_t)a.C_in, (cuuint64_t)a.C_out};
@@ -545,7 +600,7 @@ int qasr_launch_gemm_tc(qasr_ctx* ctx, const QasrConvArgs& a) {
         tmY = tmX;   // unused by the int32-output path
         tmYw = tmX;
     }
-    const size_t smem = fixed + (size_t)p.w_stages * BM * BK;
+    const size_t smem = fixed + (size_t)p.w_stages * (p.w_pair ? 2 : 1) * BM * BK;
     const int grid = p.n_items < qasr_grid_slots(ctx) ? p.n_items : qasr_grid_slots(ctx);
     QasrLaunchScope ls(ctx, QASR_K_GEMM_TC, qasr_conv_macs(a), qasr_conv_bytes(a));
     // the residual instantiation: one residual tensor beside the layer's own output, constants that keep every
