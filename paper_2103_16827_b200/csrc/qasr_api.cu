@@ -1020,9 +1020,10 @@ extern "C" int qasr_encoder_forward_host_async(qasr_ctx* ctx, const qasr_layer* 
                               lf_dev ? out_scale : nullptr);
     if (rc) return rc;
     QASR_CUDA(ctx, cudaEventRecord(ctx->ev_comp[slot], ctx->stream));
-    // the next input copy into this slot must not overtake these kernels (the host-side wait above already
-    // orders it after them; this keeps the order on the device too)
-    QASR_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_in, ctx->ev_comp[slot], 0));
+    // The next input copy into this slot cannot overtake these kernels: the call that issues it first waits, on
+    // the host, for this call's results (above). No device-side wait is put into the copy stream for it: stream
+    // order would make the OTHER slot's next input copy wait for these kernels as well, and that copy is the one
+    // that has to run beside them.
     // result copies on a third stream: they overlap the next call's kernels
     QASR_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_out, ctx->ev_comp[slot], 0));
     QASR_CUDA(ctx, cudaMemcpyAsync(logits_q_host, lq_dev, n_logit * 4, cudaMemcpyDeviceToHost, ctx->copy_out));
