@@ -1,6 +1,8 @@
 // Generic kernels: correct for any shape and alignment.  They are the path for shapes the
 // tensor-core and vectorised kernels do not take (odd sizes, stride/dilation 2, tiny channel
 // counts) and for the element-wise steps (residual add, final dequantisation).
+#include <cstring>
+
 #include "qasr_device.cuh"
 #include "sm100_ptx.cuh"
 
@@ -240,15 +242,19 @@ __global__ void __launch_bounds__(256)
 glu_vec16_kernel(const int8_t* __restrict__ x, int C, int T16, unsigned items, int q_c, const int32_t* mult,
                  const uint8_t* shift, int8_t* __restrict__ y, unsigned* status) {
     const unsigned i = blockIdx.x * blockDim.x + threadIdx.x;
+    // launched with programmatic early launch inside a layer table: the channel's constants are fetched while
+    // the kernel that writes x still runs; x is read behind the dependency wait
+    ptx::grid_dep_launch();
     if (i >= items) return;
     const unsigned t16 = i % (unsigned)T16, bc = i / (unsigned)T16;
     const unsigned c = bc % (unsigned)C, b = bc / (unsigned)C;
     const size_t row = (size_t)T16 * 16;
     const size_t ia = ((size_t)b * 2 * C + c) * row + (size_t)t16 * 16;
-    const int4 av = __ldg(reinterpret_cast<const int4*>(x + ia));
-    const int4 gv = __ldg(reinterpret_cast<const int4*>(x + ia + (size_t)C * row));
     int m, s;
     load_rq(mult, shift, (int)c, m, s, status);
+    ptx::grid_dep_wait();
+    const int4 av = __ldg(reinterpret_cast<const int4*>(x + ia));
+    const int4 gv = __ldg(reinterpret_cast<const int4*>(x + ia + (size_t)C * row));
     const int kmax = min(__clz(m) - 1, 62 - s);
     const int k = (s <= 32 && 32 - s <= kmax) ? 32 - s : max(kmax, 0);
     const int mn = m << k, sn = s + k;
@@ -271,12 +277,18 @@ glu_vec16_kernel(const int8_t* __restrict__ x, int C, int T16, unsigned items, i
 }  // namespace qasr
 
 cudaError_t qasr_launch_glu(const int8_t* x, int B, int C, int T, int q_c, const int32_t* mult,
-                            const uint8_t* shift, int8_t* y, unsigned* status, cudaStream_t st) {
+                            const uint8_t* shift, int8_t* y, unsigned* status, cudaStream_t st, int early_launch) {
     const size_t n = (size_t)B * C * T;
     if (T % 16 == 0 && (((uintptr_t)x | (uintptr_t)y) & 15u) == 0 && n / 16 < 0x7fffffffu) {
         const unsigned items = (unsigned)(n / 16);
-        qasr::glu_vec16_kernel<<<(items + 255) / 256, 256, 0, st>>>(x, C, T / 16, items, q_c, mult, shift, y, status);
-        return cudaGetLastError();
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof(cfg));
+        cfg.gridDim = dim3((items + 255) / 256); cfg.blockDim = dim3(256); cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = early_launch ? 1 : 0;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, qasr::glu_vec16_kernel, x, C, T / 16, items, q_c, mult, shift, y, status);
     }
     const unsigned blocks = (unsigned)((n + 255) / 256 < 148u * 16u ? (n + 255) / 256 : 148u * 16u);
     qasr::glu_kernel<<<blocks ? blocks : 1, 256, 0, st>>>(x, C, T, n, q_c, mult, shift, y, status);

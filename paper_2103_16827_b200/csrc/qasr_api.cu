@@ -772,7 +772,8 @@ static int enqueue_table(qasr_ctx* ctx, const qasr_layer* tb, int n, const Table
         }
         if (L.kind == QASR_LAYER_GLU) {
             QasrLaunchScope ls(ctx, QASR_K_GLU, 0, (double)B * L.C_out * T_o * 3);
-            QASR_CUDA(ctx, qasr_launch_glu(in, B, L.C_out, T_o, L.glu_qc, L.rq.mult, L.rq.shift, buf_ptr(L.out_buf), ctx->d_status, ctx->stream));
+            QASR_CUDA(ctx, qasr_launch_glu(in, B, L.C_out, T_o, L.glu_qc, L.rq.mult, L.rq.shift, buf_ptr(L.out_buf), ctx->d_status, ctx->stream,
+                                           ctx->opt_pdl ? 1 : 0));
             curC[L.out_buf] = L.C_out;
             continue;
         }

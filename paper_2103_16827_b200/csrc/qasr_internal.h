@@ -62,6 +62,6 @@ cudaError_t qasr_launch_conv_generic(const QasrConvArgs& a, unsigned* status, cu
 cudaError_t qasr_launch_residual_add(const QasrTerms& t, size_t n, int relu, int8_t* y,
                                      unsigned* status, cudaStream_t st);
 cudaError_t qasr_launch_glu(const int8_t* x, int B, int C, int T, int q_c, const int32_t* mult,
-                            const uint8_t* shift, int8_t* y, unsigned* status, cudaStream_t st);
+                            const uint8_t* shift, int8_t* y, unsigned* status, cudaStream_t st, int early_launch = 0);
 cudaError_t qasr_launch_dequant(const int32_t* acc, int B, int C, int T, const float* scale,
                                 float* out, cudaStream_t st);
