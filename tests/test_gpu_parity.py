@@ -829,6 +829,30 @@ def test_config3_jasper_full_batch_sampled_utterances(q, ctx):
     assert np.std(wq.astype(np.float64)) > 100
 
 
+@pytest.mark.parametrize("cfg,pick", [(3, [9]), (4, [5, 10])])
+def test_config3_config4_full_batch_every_layer_of_middle_utterances(q, ctx, cfg, pick):
+    """The Jasper and Conformer shapes at their full batch with a buffer of its own for every layer: every
+    intermediate tensor of middle utterances against the oracle (for config 3 that includes, at the benchmark's own
+    tile sizes, the layers whose input copy came from the previous layer's frame-major second output)."""
+    model, x = workloads.config(cfg, variant="live", unique_bufs=True)
+    wq, wf, trace = oracle.encoder_forward(model, x[pick])
+    dm = q.DeviceModel(model, 0)
+    B, _, T = x.shape
+    ws = torch.zeros(ctx.encoder_workspace_bytes(dm, B, T), dtype=torch.uint8, device="cuda")
+    last = model["layers"][-1]
+    lq = torch.zeros((B, last["C_out"], wq.shape[2]), dtype=torch.int32, device="cuda")
+    lf = torch.zeros(lq.shape, dtype=torch.float32, device="cuda")
+    ctx.encoder_forward(dm, dev(x), ws, lq, lf)
+    ctx.poll_status()
+    idx = torch.tensor(pick, device="cuda")
+    for L, o in zip(model["layers"][:-1], trace[:-1]):
+        off, C, Tl = ctx.encoder_buffer_info(dm, B, T, L["out"])
+        got = ws[off:off + B * C * Tl].view(torch.int8).reshape(B, C, Tl)[idx].cpu().numpy()
+        assert_same(got, o["y"], "config %d layer %s" % (cfg, L["name"]))
+    assert_same(lq[idx].cpu().numpy(), wq, "config %d logits_q" % cfg)
+    assert np.max(np.abs(lf[idx].cpu().numpy() - wf)) <= 1e-6
+
+
 # ------------------------------------------------------------------ no stray writes, no run-to-run differences
 GUARD = 4096
 
